@@ -1,0 +1,148 @@
+/*
+ * zipline.h - C ABI of the ZipLine barrier-selection library (CUDA, sm_100a).
+ *
+ * The operation (paper, Section III "The Problem" and Section IV "ZipLine",
+ * Algorithm 2): n workers, worker p has R predicted iteration end timestamps
+ * e^p_1 <= ... <= e^p_R.  One element is picked per worker to form Z; the
+ * waiting time is d_Z = max(Z) - min(Z); the selection returned is
+ * Z* = argmin d_Z and the next synchronisation barrier is max(Z*).  When
+ * several Z reach the minimum the earliest barrier is taken (Fig. 3 caption,
+ * "the first minimum d_Z is selected").
+ *
+ * Every entry point is extern "C", takes plain pointers and sizes, and says
+ * for each pointer whether it is host or device memory.  All device work is
+ * done by the library's own kernels; there is no CPU fallback.
+ */
+#ifndef ZIPLINE_H
+#define ZIPLINE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct zl_handle zl_handle;      /* opaque; owns device scratch only */
+
+typedef enum {
+    ZL_OK = 0,
+    ZL_ERR_INVALID_ARG = 1,   /* null/misaligned pointer, size out of range, value outside [0, 2^62) */
+    ZL_ERR_UNSUPPORTED = 2,   /* shape or magnitude the kernels cannot take (see zl_create)        */
+    ZL_ERR_NOMEM = 3,
+    ZL_ERR_CUDA = 4,          /* a CUDA runtime call failed; zl_last_cuda_error() has its code      */
+    ZL_ERR_UNSORTED = 5,      /* per instance: a row is not non-decreasing                          */
+    ZL_ERR_TIMEOUT = 6        /* per instance: an internal iteration limit was hit                  */
+} zl_status;
+
+typedef enum {
+    ZL_OBJ_RANGE = 0,  /* d_Z = max(Z) - min(Z): the paper's objective function (Section III)   */
+    ZL_OBJ_SUM = 1     /* d_Z = sum_p (max(Z) - z_p): total waiting time of all workers         */
+} zl_objective;
+
+enum {
+    ZL_FLAG_CHECK_SORTED = 1,  /* verify every row is non-decreasing (one extra pass over the input) */
+    ZL_FLAG_FULL_SWEEP = 2     /* examine every timestamp even where the search could stop early    */
+};
+
+typedef struct {
+    int32_t n_workers;     /* n >= 1                                      */
+    int32_t lookahead_R;   /* R >= 1                                      */
+    int32_t max_batch;     /* largest B passed to zl_select_batched       */
+    int32_t objective;     /* zl_objective                                */
+    int32_t device;        /* CUDA device ordinal                         */
+    int32_t flags;         /* ZL_FLAG_*                                   */
+} zl_config;
+
+/*
+ * Create a handle and allocate its device scratch for max_batch instances of
+ * n x R timestamps (Section IV: the n x R matrix M, one row per worker).
+ * cfg and out are host pointers.  ZL_ERR_UNSUPPORTED if n exceeds
+ * zl_max_workers().  The handle is not thread safe; distinct handles are
+ * independent.
+ */
+zl_status zl_create(const zl_config *cfg, zl_handle **out);
+
+/*
+ * The ZipLine search (Section IV "ZipLine", Algorithm 2) on B independent
+ * instances: merge the n sorted rows of an instance into time order (Omega),
+ * sweep it keeping the latest element of every worker (Z), evaluate d_Z
+ * wherever Z holds all n workers, keep the first minimum, then recover the
+ * chosen iteration of every worker.
+ *
+ *   d_ts      device, read only, [B][n][R] int64 microseconds, 8-byte aligned;
+ *             row p of instance b = worker p's end timestamps, non-decreasing,
+ *             every value in [0, 2^62).
+ *   B         1 .. max_batch.
+ *   d_idx     device out, [B][n] int32: 0-based index of the last iteration worker p
+ *             finishes at or before the barrier (the element of Z*).
+ *   d_barrier device out, [B] int64: max(Z*).
+ *   d_wait    device out, [B] int64: the minimum of the configured objective.
+ *   d_status  device out, [B] int32 or NULL: ZL_OK, or the per-instance error; an
+ *             instance in error gets idx = -1 and barrier = wait = INT64_MIN.
+ *   cuda_stream  a cudaStream_t (0 = default stream).  The call only enqueues work
+ *             and returns; outputs are valid once the stream has run.  It never
+ *             allocates or synchronises.  The caller owns every buffer.
+ *
+ * Result definition: wait is the minimum of d_Z over all R^n selections;
+ * barrier is the smallest max(Z) among the minimisers; idx[p] is the largest i
+ * with e^p_i <= barrier.  Returns host-detectable errors only.
+ */
+zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B,
+                            int32_t *d_idx, int64_t *d_barrier, int64_t *d_wait,
+                            int32_t *d_status, void *cuda_stream);
+
+/*
+ * The same search with HOST buffers (same shapes and meaning as above):
+ * copies the input to the device, runs the kernels, copies the results back
+ * and waits for them.  Staging buffers are allocated by the first such call
+ * on a handle (so that call allocates; later ones do not).  h_status may be
+ * NULL.  Pinned host memory makes the copies asynchronous to the host until
+ * the final wait; pageable memory works too.
+ */
+zl_status zl_select_batched_host(zl_handle *h, const int64_t *h_ts, int32_t B,
+                                 int32_t *h_idx, int64_t *h_barrier, int64_t *h_wait,
+                                 int32_t *h_status);
+
+/*
+ * Per-position intermediates of the sweep (Section IV "ZipLine": Omega sorted
+ * by value, Z updated one element per step) for B small instances, each with
+ * N = n*R <= zl_trace_max_elements().  Position k runs over Omega in
+ * (timestamp, worker, iteration) order.  All pointers are device memory,
+ * [B][N], and any of them may be NULL:
+ *   om_t/om_p/om_i  the merged order (step 1: merge)
+ *   delta, first    e^p_i - e^p_{i-1} (e^p_1 for i = 1) and first-appearance flag (step 2)
+ *   S, cnt          inclusive prefix sums of delta and first (step 3)
+ *   next, PM        e^p_{i+1} (INT64_MAX for i = R) and its exclusive prefix maximum (step 3)
+ *   d_range         max(om_t, t0, PM) - om_t, t0 = max_p e^p_1; INT64_MAX when undefined (step 4)
+ *   w_sum           n*om_t - S where cnt == n, else INT64_MAX (step 4)
+ * Asynchronous on cuda_stream; no handle, no scratch.
+ */
+zl_status zl_trace_batched(const int64_t *d_ts, int32_t B, int32_t n, int32_t R,
+                           int64_t *om_t, int32_t *om_p, int32_t *om_i,
+                           int64_t *delta, int32_t *first, int64_t *S, int32_t *cnt,
+                           int64_t *next, int64_t *PM, int64_t *d_range, int64_t *w_sum,
+                           void *cuda_stream);
+
+/* Free the scratch and the handle.  NULL is a no-op. */
+zl_status zl_destroy(zl_handle *h);
+
+/* Tuning knobs of a handle (host side; take effect at the next call).
+ * key: "threads" (128..1024, power of two), "lanes_per_row" (1..32, power of two),
+ * "segments" (time segments per instance, >= 1), "round_factor" (percent of the
+ * nominal elements per round).  0 restores the built-in choice. */
+zl_status zl_set_option(zl_handle *h, const char *key, int32_t value);
+
+/* Queries (host side). */
+const char *zl_status_string(zl_status s);
+size_t   zl_workspace_bytes(const zl_handle *h);      /* device scratch held by the handle      */
+int32_t  zl_launches_per_call(const zl_handle *h);    /* kernels one zl_select_batched enqueues  */
+int32_t  zl_segments_per_instance(const zl_handle *h, int32_t B);
+int32_t  zl_max_workers(void);                        /* largest supported n                     */
+int32_t  zl_trace_max_elements(void);                 /* largest n*R for zl_trace_batched        */
+int32_t  zl_last_cuda_error(const zl_handle *h);      /* cudaError_t of the last failed call     */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZIPLINE_H */

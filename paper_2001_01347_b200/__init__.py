@@ -1,0 +1,8 @@
+"""ZipLine barrier-selection search (ElasticBSP, arXiv 2001.01347) as sm_100a CUDA kernels.
+
+``binding`` loads ``libzipline.so`` (built in-tree by ``build``) and exposes the C ABI declared
+in ``include/zipline.h`` under the same names.
+"""
+from .binding import (ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP, ZL_OBJ_RANGE, ZL_OBJ_SUM, ZL_OK,  # noqa: F401
+                      Selection, ZipLine, ZipLineError, zl_max_workers, zl_status_string,
+                      zl_trace_batched, zl_trace_max_elements)

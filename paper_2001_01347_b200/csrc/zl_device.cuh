@@ -1,0 +1,121 @@
+// Device-side building blocks of the ZipLine kernels: key packing, block-wide
+// bitonic sort in shared memory, block-wide scans and reductions.  No CUB/Thrust.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace zl {
+
+constexpr unsigned FULL = 0xffffffffu;
+
+// ---------------------------------------------------------------------------------- keys
+// A node of the sweep is (T, V): T = time relative to the instance (tmin -> 1), V = the
+// payload the scan needs (RANGE: the same worker's next timestamp; SUM: T minus the same
+// worker's previous timestamp).  32-bit instances pack both into one 64-bit word so that the
+// sort moves a single register pair; wide instances use a 16-byte pair.
+template <typename K> struct Key;
+
+template <> struct Key<uint32_t> {
+    uint64_t w;
+    __device__ __forceinline__ static Key make(uint32_t t, uint32_t v) { return Key{((uint64_t)t << 32) | v}; }
+    __device__ __forceinline__ static Key inf() { return Key{~0ull}; }
+    __device__ __forceinline__ uint32_t t() const { return (uint32_t)(w >> 32); }
+    __device__ __forceinline__ uint32_t v() const { return (uint32_t)w; }
+    __device__ __forceinline__ bool operator>(const Key &o) const { return w > o.w; }
+};
+
+template <> struct Key<uint64_t> {
+    uint64_t a, b;
+    __device__ __forceinline__ static Key make(uint64_t t, uint64_t v) { return Key{t, v}; }
+    __device__ __forceinline__ static Key inf() { return Key{~0ull, ~0ull}; }
+    __device__ __forceinline__ uint64_t t() const { return a; }
+    __device__ __forceinline__ uint64_t v() const { return b; }
+    __device__ __forceinline__ bool operator>(const Key &o) const { return a > o.a || (a == o.a && b > o.b); }
+};
+
+template <typename K> __device__ __forceinline__ K kinf();
+template <> __device__ __forceinline__ uint32_t kinf<uint32_t>() { return 0xffffffffu; }
+template <> __device__ __forceinline__ uint64_t kinf<uint64_t>() { return ~0ull; }
+
+// ---------------------------------------------------------------------------------- sort
+// Ascending bitonic sort of keys[0..P) in shared memory, P a power of two, by the whole block.
+template <typename KeyT>
+__device__ void bitonic_sort(KeyT *keys, int P) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    for (int k = 2; k <= P; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int i = tid; i < (P >> 1); i += nt) {
+                const int lo = ((i & ~(j - 1)) << 1) | (i & (j - 1));
+                const int hi = lo | j;
+                const bool up = (lo & k) == 0;
+                KeyT x = keys[lo], y = keys[hi];
+                if ((x > y) == up) { keys[lo] = y; keys[hi] = x; }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------- scans
+struct OpMax { template <typename T> __device__ __forceinline__ T operator()(T a, T b) const { return a > b ? a : b; } };
+struct OpMin { template <typename T> __device__ __forceinline__ T operator()(T a, T b) const { return a < b ? a : b; } };
+struct OpAdd { template <typename T> __device__ __forceinline__ T operator()(T a, T b) const { return a + b; } };
+
+template <typename T> __device__ __forceinline__ T shfl_up(T v, int d) {
+    if constexpr (sizeof(T) == 8) return (T)__shfl_up_sync(FULL, (unsigned long long)v, d);
+    else return (T)__shfl_up_sync(FULL, (unsigned)v, d);
+}
+template <typename T> __device__ __forceinline__ T shfl_xor(T v, int d) {
+    if constexpr (sizeof(T) == 8) return (T)__shfl_xor_sync(FULL, (unsigned long long)v, d);
+    else return (T)__shfl_xor_sync(FULL, (unsigned)v, d);
+}
+template <typename T> __device__ __forceinline__ T shfl_idx(T v, int s) {
+    if constexpr (sizeof(T) == 8) return (T)__shfl_sync(FULL, (unsigned long long)v, s);
+    else return (T)__shfl_sync(FULL, (unsigned)v, s);
+}
+
+// One value per thread -> exclusive scan over the block in thread order (identity for thread 0)
+// and the block total.  tmp: shared, 33 elements of T.  Contains two barriers; every thread calls.
+template <typename T, typename Op>
+__device__ T block_scan_excl(T x, Op op, T identity, T *tmp, T *total) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    T inc = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        T y = shfl_up(inc, d);
+        if (lane >= d) inc = op(y, inc);
+    }
+    if (lane == 31) tmp[warp] = inc;
+    __syncthreads();
+    if (warp == 0) {
+        T w = lane < nw ? tmp[lane] : identity;
+        T winc = w;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            T y = shfl_up(winc, d);
+            if (lane >= d) winc = op(y, winc);
+        }
+        T wexc = shfl_up(winc, 1);
+        if (lane == 0) wexc = identity;
+        if (lane < nw) tmp[lane] = wexc;
+        if (lane == nw - 1) tmp[32] = winc;
+    }
+    __syncthreads();
+    T exc = shfl_up(inc, 1);
+    if (lane == 0) exc = identity;
+    exc = op(tmp[warp], exc);
+    *total = tmp[32];
+    __syncthreads();                       // tmp may be reused by the caller right away
+    return exc;
+}
+
+template <typename T, typename Op>
+__device__ __forceinline__ T warp_reduce(T x, Op op) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) x = op(x, shfl_xor(x, d));
+    return x;
+}
+
+__device__ __forceinline__ int64_t ldg64(const int64_t *p) { return (int64_t)__ldg((const long long *)p); }
+
+}  // namespace zl

@@ -1,0 +1,221 @@
+"""Parity of the CUDA path against the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as o
+import zl_inputs as zi
+from conftest import load_hand_examples
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    import paper_2001_01347_b200 as zl
+
+OBJ = [0, 1]
+
+
+def gpu_select(ts_np, objective, flags=0, options=None):
+    ts_np = np.ascontiguousarray(ts_np, dtype=np.int64)
+    B, n, R = ts_np.shape
+    h = zl.ZipLine(n, R, B, objective, 0, flags)
+    for k, v in (options or {}).items():
+        h.set_option(k, v)
+    sel = h.select_batched(torch.from_numpy(ts_np).cuda())
+    torch.cuda.synchronize()
+    h.destroy()
+    return sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()
+
+
+def assert_same(ts_np, objective, got, fn=None, which=None):
+    idx, barrier, wait, status = got
+    fn = fn or o.sweep_window
+    which = range(ts_np.shape[0]) if which is None else which
+    for b in which:
+        w, t, ix = fn(ts_np[b], objective)
+        assert status[b] == 0, (b, status[b])
+        assert (int(wait[b]), int(barrier[b])) == (w, t), (b, objective, int(wait[b]), int(barrier[b]), w, t)
+        assert (idx[b] == ix).all(), (b, idx[b][:8], ix[:8])
+
+
+# ---------------------------------------------------------------- small cases
+@pytest.mark.parametrize("objective", OBJ)
+def test_hand_examples(objective):
+    for name, M, rng_exp, sum_exp in load_hand_examples():
+        exp = rng_exp if objective == 0 else sum_exp
+        idx, barrier, wait, status = gpu_select(np.array([M]), objective)
+        assert status[0] == 0
+        assert (int(wait[0]), int(barrier[0]), idx[0].tolist()) == (exp[0], exp[1], exp[2]), name
+
+
+@pytest.mark.parametrize("objective", OBJ)
+@pytest.mark.parametrize("regime", ["dense", "sparse", "strict"])
+def test_random_tiny_vs_enumerator(objective, regime):
+    rng = np.random.default_rng(100 + objective)
+    for n, R in ((1, 1), (1, 5), (2, 2), (3, 4), (4, 5), (5, 3), (2, 9), (6, 3)):
+        B = 64
+        if regime == "dense":
+            inc, off = rng.integers(0, 4, size=(B, n, R)), rng.integers(0, 5, size=(B, n, 1))
+        elif regime == "sparse":
+            inc, off = rng.integers(0, 10 ** 9, size=(B, n, R)), rng.integers(0, 10 ** 9, size=(B, n, 1))
+        else:
+            inc, off = rng.integers(1, 50, size=(B, n, R)), rng.integers(0, 60, size=(B, n, 1))
+        ts = (off + np.cumsum(inc, axis=2)).astype(np.int64)
+        assert_same(ts, objective, gpu_select(ts, objective), fn=o.enumerate_all)
+
+
+@pytest.mark.parametrize("objective", OBJ)
+def test_ragged_medium_shapes_vs_sweep(objective):
+    # sizes that span several batches / rounds and leave ragged tails (n, R not powers of two)
+    rng = np.random.default_rng(7 + objective)
+    for n, R, B, hi in ((7, 40, 9, 1000), (33, 17, 5, 30), (100, 150, 3, 10 ** 5), (10, 150, 4, 5000),
+                        (257, 65, 2, 3), (1000, 15, 2, 200_000), (50, 1, 3, 100), (1, 300, 2, 10)):
+        inc = rng.integers(0, hi, size=(B, n, R))
+        ts = (rng.integers(0, 3 * hi, size=(B, n, 1)) + np.cumsum(inc, axis=2)).astype(np.int64)
+        assert_same(ts, objective, gpu_select(ts, objective))
+
+
+@pytest.mark.parametrize("objective", OBJ)
+def test_all_equal_and_identical_rows(objective):
+    ts = np.full((2, 37, 50), 12345, dtype=np.int64)
+    idx, barrier, wait, status = gpu_select(ts, objective)
+    assert (status == 0).all() and (wait == 0).all() and (barrier == 12345).all() and (idx == 49).all()
+    row = np.cumsum(np.arange(1, 201))
+    ts = np.broadcast_to(row, (3, 300, 200)).astype(np.int64).copy()
+    assert_same(ts, objective, gpu_select(ts, objective))
+
+
+@pytest.mark.parametrize("objective", OBJ)
+def test_uniform_shift_and_wide_spans(objective):
+    w = zi.CONFIGS["c3"].with_(B=3, n=40, R=70)
+    ts = zi.generate(w)
+    base = gpu_select(ts, objective)
+    assert_same(ts, objective, base)
+    shift = 1_700_000_000_000_000
+    idx, barrier, wait, status = gpu_select(ts + shift, objective)
+    assert (idx == base[0]).all() and (wait == base[2]).all() and (barrier == base[1] + shift).all()
+    # spans beyond 32 bits take the wide-key path
+    wide = ts * 3000
+    assert int(wide.max() - wide.min()) > 2 ** 33
+    assert_same(wide, objective, gpu_select(wide, objective))
+
+
+@pytest.mark.parametrize("objective", OBJ)
+def test_launch_shapes_do_not_change_results(objective):
+    w = zi.CONFIGS["c4"].with_(B=2, n=96, R=300)
+    ts = zi.generate(w)
+    ref = gpu_select(ts, objective)
+    assert_same(ts, objective, ref)
+    for opts in ({"segments": 7}, {"segments": 16, "threads": 128}, {"lanes_per_row": 1, "threads": 256},
+                 {"lanes_per_row": 32, "segments": 3}, {"round_factor": 5}, {"round_factor": 2000, "segments": 2}):
+        got = gpu_select(ts, objective, options=opts)
+        for a, b in zip(ref, got):
+            assert (a == b).all(), opts
+    full = gpu_select(ts, objective, flags=zl.ZL_FLAG_FULL_SWEEP, options={"segments": 5})
+    for a, b in zip(ref, full):
+        assert (a == b).all()
+
+
+# ---------------------------------------------------------------- the five workloads
+@pytest.mark.parametrize("objective", OBJ)
+def test_config_c1_vs_enumerator(objective):
+    ts = zi.generate(zi.CONFIGS["c1"])
+    assert_same(ts, objective, gpu_select(ts, objective), fn=o.enumerate_all)
+
+
+@pytest.mark.parametrize("objective", OBJ)
+def test_config_c2_full_batch(objective):
+    ts = zi.generate(zi.CONFIGS["c2"])
+    got = gpu_select(ts, objective)
+    assert_same(ts, objective, got, which=range(0, 4096, 5))
+
+
+@pytest.mark.parametrize("objective", OBJ)
+def test_config_c3_full_batch(objective):
+    ts = zi.generate(zi.CONFIGS["c3"])
+    got = gpu_select(ts, objective)
+    assert_same(ts, objective, got, which=range(0, 1024, 16))
+
+
+@pytest.mark.parametrize("objective", OBJ)
+def test_config_c4_full_batch(objective):
+    ts = zi.generate(zi.CONFIGS["c4"])
+    got = gpu_select(ts, objective)
+    assert (got[3] == 0).all()
+    assert_same(ts, objective, got, which=range(0, 64, 8))
+
+
+@pytest.mark.parametrize("objective", OBJ)
+def test_config_c5_full_batch(objective):
+    ts = zi.generate(zi.CONFIGS["c5"])
+    got = gpu_select(ts, objective)
+    assert (got[3] == 0).all()
+    assert_same(ts, objective, got, which=[0, 5])
+    # properties that hold for every instance at any size
+    idx, barrier, wait, _ = got
+    for b in range(ts.shape[0]):
+        chosen = ts[b][np.arange(ts.shape[1]), idx[b]]
+        assert chosen.max() == barrier[b] and (chosen <= barrier[b]).all()
+        assert wait[b] == (barrier[b] - chosen.min() if objective == 0 else (barrier[b] - chosen).sum())
+
+
+# ---------------------------------------------------------------- errors and flags
+def test_per_instance_errors():
+    ts = np.cumsum(np.ones((3, 4, 6), dtype=np.int64), axis=2) * 10
+    ts[1, 2, 3] = 5                      # row 2 of instance 1 goes backwards
+    idx, barrier, wait, status = gpu_select(ts, 0, flags=zl.ZL_FLAG_CHECK_SORTED)
+    assert status.tolist() == [0, zl.binding.ZL_ERR_UNSORTED, 0]
+    assert (idx[1] == -1).all() and barrier[1] == np.iinfo(np.int64).min and wait[1] == np.iinfo(np.int64).min
+    assert_same(ts, 0, (idx, barrier, wait, status), which=[0, 2])
+    ts2 = ts.copy()
+    ts2[1] = ts[0]
+    ts2[2, 0, 0] = -4                    # negative timestamp
+    idx, barrier, wait, status = gpu_select(ts2, 0)
+    assert status.tolist() == [0, 0, zl.binding.ZL_ERR_INVALID_ARG]
+
+
+def test_host_detected_errors():
+    with pytest.raises(zl.ZipLineError):
+        zl.ZipLine(zl.zl_max_workers() + 1, 4, 1)
+    with pytest.raises(zl.ZipLineError):
+        zl.ZipLine(0, 4, 1)
+    h = zl.ZipLine(4, 4, 2)
+    ts = torch.zeros((3, 4, 4), dtype=torch.int64, device="cuda")
+    with pytest.raises(zl.ZipLineError):
+        h.select_batched(ts)             # B > max_batch
+    with pytest.raises(zl.ZipLineError):
+        h.set_option("no_such_option", 1)
+    assert h.launches_per_call == 3 and h.workspace_bytes > 0
+    h.destroy()
+
+
+def test_host_buffer_entry_point_and_streams():
+    w = zi.CONFIGS["c2"].with_(B=64)
+    ts = zi.generate(w)
+    h = zl.ZipLine(w.n, w.R, 64, 0)
+    pinned = torch.from_numpy(ts).pin_memory()
+    sel = h.select_batched_host(pinned)
+    assert_same(ts, 0, (sel.idx.numpy(), sel.barrier.numpy(), sel.wait.numpy(), sel.status.numpy()))
+    s = torch.cuda.Stream()
+    d = torch.from_numpy(ts).cuda()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        sel2 = h.select_batched(d[:10])
+    s.synchronize()
+    assert (sel2.wait.cpu() == sel.wait[:10]).all() and (sel2.idx.cpu() == sel.idx[:10]).all()
+    h.destroy()
+
+
+# ---------------------------------------------------------------- per-step intermediates
+def test_trace_matches_oracle_trace():
+    rng = np.random.default_rng(17)
+    for n, R, hi in ((4, 8, 50), (16, 64, 10 ** 6), (7, 33, 3), (1, 20, 10), (30, 1, 10), (64, 64, 100)):
+        B = 5
+        inc = rng.integers(0, hi, size=(B, n, R))
+        ts = (rng.integers(0, 3 * hi, size=(B, n, 1)) + np.cumsum(inc, axis=2)).astype(np.int64)
+        tr = zl.zl_trace_batched(torch.from_numpy(ts).cuda())
+        torch.cuda.synchronize()
+        for b in range(B):
+            ref = o.trace(ts[b])
+            for k in ref:
+                assert (tr[k][b].cpu().numpy() == ref[k]).all(), (k, n, R, b)
