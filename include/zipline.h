@@ -124,6 +124,18 @@ zl_status zl_trace_batched(const int64_t *d_ts, int32_t B, int32_t n, int32_t R,
                            int64_t *next, int64_t *PM, int64_t *d_range, int64_t *w_sum,
                            void *cuda_stream);
 
+/*
+ * Optional per-kernel timing (no counterpart in the paper; a measurement aid).
+ * After zl_profile_begin(h, max_calls) every zl_select_batched on h records CUDA
+ * events on the caller's stream around its three stages, for up to max_calls calls.
+ * zl_profile_read waits for the recorded calls, returns their number and the summed
+ * milliseconds of the prologue, sweep and finalize kernels, and clears the record.
+ * zl_profile_end releases the events.  All pointers are host pointers.
+ */
+zl_status zl_profile_begin(zl_handle *h, int32_t max_calls);
+zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_prologue, float *ms_sweep, float *ms_finalize);
+zl_status zl_profile_end(zl_handle *h);
+
 /* Free the scratch and the handle.  NULL is a no-op. */
 zl_status zl_destroy(zl_handle *h);
 

@@ -20,7 +20,8 @@ ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP = 1, 2
 
 EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace_batched", "zl_destroy",
            "zl_set_option", "zl_status_string", "zl_workspace_bytes", "zl_launches_per_call",
-           "zl_segments_per_instance", "zl_max_workers", "zl_trace_max_elements", "zl_last_cuda_error")
+           "zl_segments_per_instance", "zl_max_workers", "zl_trace_max_elements", "zl_last_cuda_error",
+           "zl_profile_begin", "zl_profile_read", "zl_profile_end")
 
 
 class zl_config(ctypes.Structure):
@@ -44,9 +45,13 @@ def _load() -> ctypes.CDLL:
     lib.zl_launches_per_call.argtypes = [vp]
     lib.zl_segments_per_instance.argtypes = [vp, i32]
     lib.zl_last_cuda_error.argtypes = [vp]
+    lib.zl_profile_begin.argtypes = [vp, i32]
+    lib.zl_profile_read.argtypes = [vp, vp, vp, vp, vp]
+    lib.zl_profile_end.argtypes = [vp]
     for name in ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace_batched", "zl_destroy",
                  "zl_set_option", "zl_launches_per_call", "zl_segments_per_instance", "zl_max_workers",
-                 "zl_trace_max_elements", "zl_last_cuda_error"):
+                 "zl_trace_max_elements", "zl_last_cuda_error", "zl_profile_begin", "zl_profile_read",
+                 "zl_profile_end"):
         getattr(lib, name).restype = ctypes.c_int
     return lib
 
@@ -139,6 +144,19 @@ class ZipLine:
                                         out.wait.data_ptr(), out.status.data_ptr())
         _check(rc, "zl_select_batched_host")
         return out
+
+    def profile_begin(self, max_calls: int):
+        _check(lib.zl_profile_begin(self._h, int(max_calls)), "zl_profile_begin")
+
+    def profile_read(self) -> dict:
+        calls = ctypes.c_int32()
+        a, b, c = ctypes.c_float(), ctypes.c_float(), ctypes.c_float()
+        _check(lib.zl_profile_read(self._h, ctypes.addressof(calls), ctypes.addressof(a), ctypes.addressof(b),
+                                   ctypes.addressof(c)), "zl_profile_read")
+        return {"calls": calls.value, "ms_prologue": a.value, "ms_sweep": b.value, "ms_finalize": c.value}
+
+    def profile_end(self):
+        _check(lib.zl_profile_end(self._h), "zl_profile_end")
 
     def set_option(self, key: str, value: int):
         _check(lib.zl_set_option(self._h, key.encode(), int(value)), f"zl_set_option({key})")

@@ -548,6 +548,9 @@ struct zl_handle {
     int opt_threads, opt_lanes, opt_segments, opt_round_factor;
     int last_cuda_error;
     int launches;
+    // optional per-kernel timing: 4 events per recorded call
+    cudaEvent_t *prof_ev;
+    int prof_cap, prof_calls;
 };
 
 namespace {
@@ -652,12 +655,61 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     return ZL_OK;
 }
 
+zl_status zl_profile_end(zl_handle *h) {
+    if (!h) return ZL_ERR_INVALID_ARG;
+    if (h->prof_ev) {
+        for (int i = 0; i < 4 * h->prof_cap; ++i) cudaEventDestroy(h->prof_ev[i]);
+        delete[] h->prof_ev;
+    }
+    h->prof_ev = nullptr;
+    h->prof_cap = h->prof_calls = 0;
+    return ZL_OK;
+}
+
+zl_status zl_profile_begin(zl_handle *h, int32_t max_calls) {
+    if (!h || max_calls < 1 || max_calls > 65536) return ZL_ERR_INVALID_ARG;
+    zl_profile_end(h);
+    ZL_CUDA(h, cudaSetDevice(h->cfg.device));
+    h->prof_ev = new (std::nothrow) cudaEvent_t[4 * (size_t)max_calls];
+    if (!h->prof_ev) return ZL_ERR_NOMEM;
+    for (int i = 0; i < 4 * max_calls; ++i) {
+        cudaError_t e = cudaEventCreate(&h->prof_ev[i]);
+        if (e != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(h->prof_ev[j]);
+            delete[] h->prof_ev;
+            h->prof_ev = nullptr;
+            return cuda_fail(h, e);
+        }
+    }
+    h->prof_cap = max_calls;
+    h->prof_calls = 0;
+    return ZL_OK;
+}
+
+zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_prologue, float *ms_sweep, float *ms_finalize) {
+    if (!h || !calls || !ms_prologue || !ms_sweep || !ms_finalize) return ZL_ERR_INVALID_ARG;
+    *calls = h->prof_calls;
+    *ms_prologue = *ms_sweep = *ms_finalize = 0.f;
+    for (int c = 0; c < h->prof_calls; ++c) {
+        cudaEvent_t *ev = h->prof_ev + 4 * (size_t)c;
+        ZL_CUDA(h, cudaEventSynchronize(ev[3]));
+        float a = 0.f, b = 0.f, d = 0.f;
+        ZL_CUDA(h, cudaEventElapsedTime(&a, ev[0], ev[1]));
+        ZL_CUDA(h, cudaEventElapsedTime(&b, ev[1], ev[2]));
+        ZL_CUDA(h, cudaEventElapsedTime(&d, ev[2], ev[3]));
+        *ms_prologue += a; *ms_sweep += b; *ms_finalize += d;
+    }
+    h->prof_calls = 0;
+    return ZL_OK;
+}
+
 zl_status zl_destroy(zl_handle *h) {
     if (!h) return ZL_OK;
     cudaSetDevice(h->cfg.device);
     cudaFree(h->d_meta); cudaFree(h->d_seg);
     cudaFree(h->s_ts); cudaFree(h->s_idx); cudaFree(h->s_barrier); cudaFree(h->s_wait); cudaFree(h->s_status);
     if (h->s_stream) cudaStreamDestroy(h->s_stream);
+    zl_profile_end(h);
     delete h;
     return ZL_OK;
 }
@@ -700,6 +752,8 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     const LaunchPlan p = make_plan(h, B);
     if (p.smem > 200 * 1024) return ZL_ERR_UNSUPPORTED;
 
+    cudaEvent_t *ev = (h->prof_ev && h->prof_calls < h->prof_cap) ? h->prof_ev + 4 * (size_t)h->prof_calls : nullptr;
+    if (ev) cudaEventRecord(ev[0], st);
     zl::k_prologue<<<B, 256, 0, st>>>(d_ts, n, R, obj, h->d_meta);
     if (h->cfg.flags & ZL_FLAG_CHECK_SORTED) {
         const size_t total = (size_t)B * n * R;
@@ -710,9 +764,12 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     sp.ts = d_ts; sp.meta = h->d_meta; sp.seg = h->d_seg;
     sp.n = n; sp.R = R; sp.nseg = p.nseg; sp.G = p.G; sp.cap = p.cap; sp.flags = h->cfg.flags; sp.target = p.target;
     const dim3 grid(p.nseg, B);
+    if (ev) cudaEventRecord(ev[1], st);
     if (obj == ZL_OBJ_RANGE) zl::k_sweep<ZL_OBJ_RANGE><<<grid, p.threads, p.smem, st>>>(sp);
     else zl::k_sweep<ZL_OBJ_SUM><<<grid, p.threads, p.smem, st>>>(sp);
+    if (ev) cudaEventRecord(ev[2], st);
     zl::k_finalize<<<B, 256, 0, st>>>(d_ts, n, R, p.nseg, obj, h->d_meta, h->d_seg, d_idx, d_barrier, d_wait, d_status);
+    if (ev) { cudaEventRecord(ev[3], st); ++h->prof_calls; }
     ZL_CUDA(h, cudaGetLastError());
     h->launches += zl_launches_per_call(h);
     return ZL_OK;
