@@ -136,6 +136,46 @@ zl_status zl_profile_begin(zl_handle *h, int32_t max_calls);
 zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_prologue, float *ms_sweep, float *ms_finalize);
 zl_status zl_profile_end(zl_handle *h);
 
+/*
+ * The same search without a handle and without any allocation (the paper has no
+ * counterpart; this exists for callers that cannot allocate device memory).
+ *
+ * Some programs may not call cudaMalloc where they need a barrier decision: a
+ * parameter-server thread that runs inside a process whose framework has already
+ * claimed all device memory for its own pool, a service with a fixed memory budget
+ * that forbids allocation after start-up, or a latency-critical loop that must not
+ * take the driver's allocation lock (cudaMalloc and cudaFree can stall every stream
+ * of the device).  zl_create allocates the search's scratch (per-instance summaries
+ * and per-segment partial results) with cudaMalloc; this entry point keeps that
+ * scratch in a fixed array compiled into the library instead, zl_noalloc_scratch_bytes()
+ * bytes (about 400 KB) that every GPU using the library holds until the process exits.
+ * It calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * Arguments are those of zl_create's configuration (n_workers, lookahead_R, objective,
+ * flags) followed by those of zl_select_batched, with the same meaning, layout and
+ * ownership; the device is the calling thread's current CUDA device, which must own
+ * every buffer.  Asynchronous on cuda_stream.
+ *
+ * Limits: B <= zl_noalloc_max_batch() (256), and B times the number of time segments
+ * the launch planner picks must fit the array; larger requests return
+ * ZL_ERR_UNSUPPORTED with a message on stderr and launch nothing.
+ *
+ * First call on a device: looks up the array's device address and raises the sweep
+ * kernel's shared-memory limit.  Make that first call outside any stream capture.
+ *
+ * Sharing: every call on a device uses the one array, which keeps whatever the last
+ * call left there.  Nothing in it has to be cleared (each call rewrites all the
+ * records it reads), but two calls whose kernels overlap on the GPU - different
+ * streams, or different host threads - race on it and give wrong results.  Issue
+ * them on one stream, or order them with events.
+ */
+zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int32_t objective, int32_t flags,
+                                    const int64_t *d_ts, int32_t B,
+                                    int32_t *d_idx, int64_t *d_barrier, int64_t *d_wait,
+                                    int32_t *d_status, void *cuda_stream);
+int32_t  zl_noalloc_max_batch(void);       /* largest B of zl_select_batched_noalloc           */
+size_t   zl_noalloc_scratch_bytes(void);   /* size of the fixed device array it works in       */
+
 /* Free the scratch and the handle.  NULL is a no-op. */
 zl_status zl_destroy(zl_handle *h);
 

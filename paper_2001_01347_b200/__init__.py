@@ -5,4 +5,5 @@ in ``include/zipline.h`` under the same names.
 """
 from .binding import (ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP, ZL_OBJ_RANGE, ZL_OBJ_SUM, ZL_OK,  # noqa: F401
                       Selection, ZipLine, ZipLineError, zl_max_workers, zl_status_string,
+                      zl_noalloc_max_batch, zl_noalloc_scratch_bytes, zl_select_batched_noalloc,
                       zl_trace_batched, zl_trace_max_elements)

@@ -21,7 +21,8 @@ ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP = 1, 2
 EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace_batched", "zl_destroy",
            "zl_set_option", "zl_status_string", "zl_workspace_bytes", "zl_launches_per_call",
            "zl_segments_per_instance", "zl_max_workers", "zl_trace_max_elements", "zl_last_cuda_error",
-           "zl_profile_begin", "zl_profile_read", "zl_profile_end")
+           "zl_profile_begin", "zl_profile_read", "zl_profile_end",
+           "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes")
 
 
 class zl_config(ctypes.Structure):
@@ -48,6 +49,10 @@ def _load() -> ctypes.CDLL:
     lib.zl_profile_begin.argtypes = [vp, i32]
     lib.zl_profile_read.argtypes = [vp, vp, vp, vp, vp]
     lib.zl_profile_end.argtypes = [vp]
+    lib.zl_select_batched_noalloc.argtypes = [i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
+    lib.zl_select_batched_noalloc.restype = ctypes.c_int
+    lib.zl_noalloc_max_batch.restype = ctypes.c_int
+    lib.zl_noalloc_scratch_bytes.restype = ctypes.c_size_t
     for name in ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace_batched", "zl_destroy",
                  "zl_set_option", "zl_launches_per_call", "zl_segments_per_instance", "zl_max_workers",
                  "zl_trace_max_elements", "zl_last_cuda_error", "zl_profile_begin", "zl_profile_read",
@@ -186,6 +191,31 @@ class ZipLine:
             self.destroy()
         except Exception:
             pass
+
+
+def zl_noalloc_max_batch() -> int:
+    return lib.zl_noalloc_max_batch()
+
+
+def zl_noalloc_scratch_bytes() -> int:
+    return lib.zl_noalloc_scratch_bytes()
+
+
+def zl_select_batched_noalloc(ts: torch.Tensor, out: Selection, objective: int = ZL_OBJ_RANGE, flags: int = 0,
+                              stream: torch.cuda.Stream | None = None) -> Selection:
+    """The search through the entry point that allocates nothing: no handle, scratch in the library's
+    fixed device array.  ``ts`` is CUDA int64 [B, n, R] on the current device and ``out`` holds the
+    caller's result tensors (this wrapper allocates nothing either).  Calls that overlap on the GPU
+    race on the shared array; keep them on one stream."""
+    B, n, R = ts.shape
+    s = stream if stream is not None else torch.cuda.current_stream(ts.device)
+    rc = lib.zl_select_batched_noalloc(n, R, objective, flags, _dev_ptr(ts, torch.int64, B * n * R, "ts"), B,
+                                       _dev_ptr(out.idx, torch.int32, B * n, "idx"),
+                                       _dev_ptr(out.barrier, torch.int64, B, "barrier"),
+                                       _dev_ptr(out.wait, torch.int64, B, "wait"),
+                                       _dev_ptr(out.status, torch.int32, B, "status"), s.cuda_stream)
+    _check(rc, "zl_select_batched_noalloc")
+    return out
 
 
 TRACE_FIELDS = (("om_t", torch.int64), ("om_p", torch.int32), ("om_i", torch.int32), ("delta", torch.int64),

@@ -16,6 +16,7 @@
 #include <stdio.h>
 #include <string.h>
 #include <algorithm>
+#include <mutex>
 #include <new>
 
 #include "../../include/zipline.h"
@@ -812,6 +813,98 @@ zl_status zl_trace_batched(const int64_t *d_ts, int32_t B, int32_t n, int32_t R,
     cudaError_t e = cudaFuncSetAttribute(zl::k_trace, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(zl::TRACE_MAX * sizeof(zl::TKey)));
     if (e != cudaSuccess) return ZL_ERR_CUDA;
     zl::k_trace<<<B, 256, smem, (cudaStream_t)cuda_stream>>>(d_ts, n, R, om_t, om_p, om_i, delta, first, S, cnt, next, PM, d_range, w_sum);
+    return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------ no-allocation entry point
+// Scratch for zl_select_batched_noalloc lives in this fixed device array instead of a handle's
+// cudaMalloc'ed buffers.  Layout: NOALLOC_MAX_BATCH InstMeta records, then NOALLOC_MAX_SEGS SegResult
+// records.  Every GPU that loads the library holds these bytes until the process exits.
+namespace {
+constexpr int NOALLOC_MAX_BATCH = 256;
+constexpr int NOALLOC_MAX_SEGS = 16384;                       // B * (time segments per instance) of one call
+constexpr size_t NOALLOC_META_BYTES = (size_t)NOALLOC_MAX_BATCH * sizeof(zl::InstMeta);
+constexpr size_t NOALLOC_BYTES = NOALLOC_META_BYTES + (size_t)NOALLOC_MAX_SEGS * sizeof(zl::SegResult);
+static_assert(NOALLOC_META_BYTES % 256 == 0, "segment records must start on a 256-byte boundary");
+constexpr int NOALLOC_MAX_DEVICES = 64;
+}  // namespace
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+
+namespace {
+std::mutex g_noalloc_mutex;
+void *g_noalloc_ptr[NOALLOC_MAX_DEVICES];                     // device address of the array, per device
+int g_noalloc_sms[NOALLOC_MAX_DEVICES];
+}  // namespace
+
+int32_t zl_noalloc_max_batch(void) { return NOALLOC_MAX_BATCH; }
+size_t zl_noalloc_scratch_bytes(void) { return NOALLOC_BYTES; }
+
+zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int32_t objective, int32_t flags,
+                                    const int64_t *d_ts, int32_t B, int32_t *d_idx, int64_t *d_barrier,
+                                    int64_t *d_wait, int32_t *d_status, void *cuda_stream) {
+    if (!d_ts || !d_idx || !d_barrier || !d_wait) return ZL_ERR_INVALID_ARG;
+    if (n_workers < 1 || lookahead_R < 1 || B < 1) return ZL_ERR_INVALID_ARG;
+    if (objective != ZL_OBJ_RANGE && objective != ZL_OBJ_SUM) return ZL_ERR_INVALID_ARG;
+    if (flags & ~(ZL_FLAG_CHECK_SORTED | ZL_FLAG_FULL_SWEEP)) return ZL_ERR_INVALID_ARG;
+    if (((uintptr_t)d_ts & 7) || ((uintptr_t)d_barrier & 7) || ((uintptr_t)d_wait & 7) || ((uintptr_t)d_idx & 3) ||
+        ((uintptr_t)d_status & 3))
+        return ZL_ERR_INVALID_ARG;
+    if (n_workers > zl::MAX_WORKERS || (long long)n_workers * lookahead_R > (1LL << 31) - 1) return ZL_ERR_UNSUPPORTED;
+    if (B > NOALLOC_MAX_BATCH) {
+        fprintf(stderr, "zl_select_batched_noalloc: B = %d exceeds the fixed scratch (at most %d instances per call)\n",
+                B, NOALLOC_MAX_BATCH);
+        return ZL_ERR_UNSUPPORTED;
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= NOALLOC_MAX_DEVICES) return ZL_ERR_CUDA;
+
+    // a handle on the stack carries the shape to the launch planner; nothing is allocated for it
+    zl_handle tmp;
+    memset(&tmp, 0, sizeof(tmp));
+    tmp.cfg.n_workers = n_workers; tmp.cfg.lookahead_R = lookahead_R; tmp.cfg.max_batch = B;
+    tmp.cfg.objective = objective; tmp.cfg.device = dev; tmp.cfg.flags = flags;
+    {
+        // once per device, with that device current: the array's name is only a host-side stand-in, the
+        // kernels need the address the runtime reports for it
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_ptr[dev]) {
+            void *ptr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress((void **)&ptr, g_noalloc_scratch);
+            if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_noalloc_sms[dev], cudaDevAttrMultiProcessorCount, dev);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e != cudaSuccess || !ptr) return ZL_ERR_CUDA;
+            g_noalloc_ptr[dev] = ptr;
+        }
+        tmp.num_sms = g_noalloc_sms[dev];
+    }
+    const LaunchPlan p = make_plan(&tmp, B);
+    if (p.smem > 200 * 1024) return ZL_ERR_UNSUPPORTED;
+    if ((long long)B * p.nseg > NOALLOC_MAX_SEGS) {
+        fprintf(stderr, "zl_select_batched_noalloc: %d instances x %d time segments exceed the fixed scratch (%d records)\n",
+                B, p.nseg, NOALLOC_MAX_SEGS);
+        return ZL_ERR_UNSUPPORTED;
+    }
+    zl::InstMeta *meta = (zl::InstMeta *)g_noalloc_ptr[dev];
+    zl::SegResult *seg = (zl::SegResult *)((unsigned char *)g_noalloc_ptr[dev] + NOALLOC_META_BYTES);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // Nothing in the scratch has to start at zero: the prologue rewrites every InstMeta of this call and
+    // every sweep CTA rewrites its SegResult before finalize reads them, so the last call's contents are
+    // never read.
+    zl::k_prologue<<<B, 256, 0, st>>>(d_ts, n_workers, lookahead_R, objective, meta);
+    if (flags & ZL_FLAG_CHECK_SORTED) {
+        const size_t total = (size_t)B * n_workers * lookahead_R;
+        const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)tmp.num_sms * 16);
+        zl::k_check_sorted<<<blocks, 256, 0, st>>>(d_ts, n_workers, lookahead_R, total, meta);
+    }
+    zl::SweepParams sp;
+    sp.ts = d_ts; sp.meta = meta; sp.seg = seg;
+    sp.n = n_workers; sp.R = lookahead_R; sp.nseg = p.nseg; sp.G = p.G; sp.cap = p.cap; sp.flags = flags; sp.target = p.target;
+    const dim3 grid(p.nseg, B);
+    if (objective == ZL_OBJ_RANGE) zl::k_sweep<ZL_OBJ_RANGE><<<grid, p.threads, p.smem, st>>>(sp);
+    else zl::k_sweep<ZL_OBJ_SUM><<<grid, p.threads, p.smem, st>>>(sp);
+    zl::k_finalize<<<B, 256, 0, st>>>(d_ts, n_workers, lookahead_R, p.nseg, objective, meta, seg, d_idx, d_barrier, d_wait, d_status);
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;
 }
 
