@@ -261,17 +261,23 @@ def main():
     peak, peak_kind = measured_peak_gbs()
     lmin = ts_np[:, :, -1].min(axis=1)
     examined = int((ts_np <= lmin[:, None, None]).sum()) if objective == 0 else nts
-    sweep_ms = prof["ms_sweep"] / prof["calls"]
+    def dominant(pr):
+        stages = {"k_prologue": pr["ms_prologue"], "k_filter": pr["ms_filter"], "k_small+k_sweep": pr["ms_sweep"],
+                  "k_finalize": pr["ms_finalize"]}
+        name = max(stages, key=stages.get)
+        return name, stages[name] / pr["calls"]
+
+    dom, sweep_ms = dominant(prof)
     ach = examined * 8 / (sweep_ms * 1e-3) / 1e9
-    sweep_ms_f = prof_f["ms_sweep"] / prof_f["calls"]
+    dom_f, sweep_ms_f = dominant(prof_f)
     ach_f = nts * 8 / (sweep_ms_f * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "k_sweep", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
                 "peak_kind": f"{peak_kind} copy bandwidth", "traffic": None,
                 "bytes_per_launch": examined * 8, "ms_per_launch": sweep_ms,
                 "bytes_model": "8 B per timestamp not after the first exhausted row (the search stops there)"
                 if objective == 0 else "8 B per timestamp"}
     full = {"value": nts / (ms_f / steps_f * 1e-3), "unit": "timestamps/s", "ms_per_step": ms_f / steps_f,
-            "roofline": {"bound": "hbm", "kernel": "k_sweep", "achieved": ach_f, "peak": peak, "unit": "GB/s",
+            "roofline": {"bound": "hbm", "kernel": dom_f, "achieved": ach_f, "peak": peak, "unit": "GB/s",
                          "frac": ach_f / peak, "bytes_per_launch": nts * 8, "ms_per_launch": sweep_ms_f, "traffic": None}}
 
     cpu = None
@@ -283,8 +289,9 @@ def main():
     cfg = workload_config(w, objective, world)
     cfg.update({"selections_per_s": world * w.B / (ms_step * 1e-3), "early_stop": objective == 0,
                 "examined_fraction": examined / nts, "segments_per_instance": None,
-                "kernel_ms": {"prologue": prof["ms_prologue"] / prof["calls"], "sweep": sweep_ms,
-                              "finalize": prof["ms_finalize"] / prof["calls"]},
+                "kernel_ms": {k[3:]: prof[k] / prof["calls"] for k in ("ms_prologue", "ms_filter", "ms_sweep", "ms_finalize")},
+                "kernel_ms_full_sweep": {k[3:]: prof_f[k] / prof_f["calls"]
+                                         for k in ("ms_prologue", "ms_filter", "ms_sweep", "ms_finalize")},
                 "all_status_ok": status_ok, "options": args.opt})
     line = {"metric": METRIC, "value": value, "unit": "timestamps/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",

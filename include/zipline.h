@@ -125,15 +125,17 @@ zl_status zl_trace_batched(const int64_t *d_ts, int32_t B, int32_t n, int32_t R,
                            void *cuda_stream);
 
 /*
- * Optional per-kernel timing (no counterpart in the paper; a measurement aid).
+ * Optional per-stage timing (no counterpart in the paper; a measurement aid).
  * After zl_profile_begin(h, max_calls) every zl_select_batched on h records CUDA
- * events on the caller's stream around its three stages, for up to max_calls calls.
- * zl_profile_read waits for the recorded calls, returns their number and the summed
- * milliseconds of the prologue, sweep and finalize kernels, and clears the record.
- * zl_profile_end releases the events.  All pointers are host pointers.
+ * events on the caller's stream between its stages, for up to max_calls calls.
+ * zl_profile_read waits for the recorded calls, returns their number and, in
+ * ms_stage[0..3], the summed milliseconds of: prologue (column scans, filter table),
+ * filter pass, sort + sweep (the filtered-list kernel and the segment sweep kernel),
+ * finalize; it then clears the record.  zl_profile_end releases the events.
+ * All pointers are host pointers.
  */
 zl_status zl_profile_begin(zl_handle *h, int32_t max_calls);
-zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_prologue, float *ms_sweep, float *ms_finalize);
+zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_stage);
 zl_status zl_profile_end(zl_handle *h);
 
 /*
@@ -182,7 +184,8 @@ zl_status zl_destroy(zl_handle *h);
 /* Tuning knobs of a handle (host side; take effect at the next call).
  * key: "threads" (128..1024, power of two), "lanes_per_row" (1..32, power of two),
  * "segments" (time segments per instance, >= 1), "round_factor" (percent of the
- * nominal elements per round).  0 restores the built-in choice. */
+ * nominal elements per round), "no_filter" (1: RANGE skips the filter pass and sweeps
+ * every instance by time segments).  0 restores the built-in choice. */
 zl_status zl_set_option(zl_handle *h, const char *key, int32_t value);
 
 /* Queries (host side). */

@@ -47,7 +47,7 @@ def _load() -> ctypes.CDLL:
     lib.zl_segments_per_instance.argtypes = [vp, i32]
     lib.zl_last_cuda_error.argtypes = [vp]
     lib.zl_profile_begin.argtypes = [vp, i32]
-    lib.zl_profile_read.argtypes = [vp, vp, vp, vp, vp]
+    lib.zl_profile_read.argtypes = [vp, vp, vp]
     lib.zl_profile_end.argtypes = [vp]
     lib.zl_select_batched_noalloc.argtypes = [i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
     lib.zl_select_batched_noalloc.restype = ctypes.c_int
@@ -155,10 +155,9 @@ class ZipLine:
 
     def profile_read(self) -> dict:
         calls = ctypes.c_int32()
-        a, b, c = ctypes.c_float(), ctypes.c_float(), ctypes.c_float()
-        _check(lib.zl_profile_read(self._h, ctypes.addressof(calls), ctypes.addressof(a), ctypes.addressof(b),
-                                   ctypes.addressof(c)), "zl_profile_read")
-        return {"calls": calls.value, "ms_prologue": a.value, "ms_sweep": b.value, "ms_finalize": c.value}
+        ms = (ctypes.c_float * 4)()
+        _check(lib.zl_profile_read(self._h, ctypes.addressof(calls), ctypes.addressof(ms)), "zl_profile_read")
+        return {"calls": calls.value, "ms_prologue": ms[0], "ms_filter": ms[1], "ms_sweep": ms[2], "ms_finalize": ms[3]}
 
     def profile_end(self):
         _check(lib.zl_profile_end(self._h), "zl_profile_end")

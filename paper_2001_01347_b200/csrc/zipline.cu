@@ -36,6 +36,10 @@ struct InstMeta {
     uint64_t tend;       // max_p e^p_R, relative  (= span + 1)
     int32_t status;      // zl_status of the instance
     int32_t use32;       // relative times fit 32 bits
+    uint32_t sh;         // filter table: cell c covers relative times [1 + (c << sh), 1 + ((c + 1) << sh))
+    uint32_t ncell;      // cells in use (0: the instance does not take the filter path)
+    uint32_t count;      // survivors appended by the filter pass (may run past the list capacity)
+    uint32_t pad;
 };
 
 struct SegResult {
@@ -50,37 +54,57 @@ struct SweepParams {
     InstMeta *meta;
     SegResult *seg;
     int32_t n, R, nseg, G, cap, flags, target;
+    uint32_t listcap;    // > 0: instances whose filtered list fits are handled by k_small, not here
 };
 
+// An instance goes through the filter + small-sort path when it has a table and its survivors fit the list.
+__device__ __forceinline__ bool handled_by_filter(const InstMeta &M, uint32_t listcap) {
+    return listcap > 0 && M.ncell > 0 && M.count <= listcap;
+}
+
 // ------------------------------------------------------------------------------ prologue
-__global__ void __launch_bounds__(256) k_prologue(const int64_t *ts, int n, int R, int objective, InstMeta *meta) {
-    const int b = blockIdx.x;
+// Column scans per instance, and (RANGE, 32-bit instances) the filter table.
+//
+// Filter table.  For the RANGE objective an element e matters only if next(e) > G(T(e)), where
+// G(t) = max(t, t0, max{next(e') : T(e') < t}) is max(Z) of the best Z whose minimum is at time t:
+//   - if next(e) <= G(T(e)) the element cannot raise the running maximum, so PM of every later
+//     element is unchanged without it;
+//   - and it is not needed as a candidate: moving min(Z) from e to the next element in time keeps
+//     max(Z) and shrinks d_Z (or, among equal times, another element of the group qualifies).
+// Any lower bound L(t) <= G(t) therefore gives an exact filter "keep e iff next(e) > max(T, L(T))".
+// The table holds, per time cell c, L = max(t0, max over a few slow rows p of the first element of p
+// at or after the cell's start) - every such element is next(e') of an element before the cell, or a
+// first element (<= t0).  Slow rows (long iterations) are the ones that set G most of the time.
+constexpr int FILTER_ROWS = 32;      // rows that build the table
+constexpr int FILTER_MAX_CELLS = 8192;
+
+__global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int R, int objective, int flags,
+                                                    InstMeta *meta, uint32_t *table_all, int max_cells) {
+    const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
     const int64_t *inst = ts + (size_t)b * n * R;
-    int64_t mn1 = INT64_MAX, mx1 = INT64_MIN, mnR = INT64_MAX, mxR = INT64_MIN;
-    for (int p = threadIdx.x; p < n; p += blockDim.x) {
-        int64_t e1 = ldg64(inst + (size_t)p * R), eR = ldg64(inst + (size_t)p * R + R - 1);
+    __shared__ uint64_t s[4][32];
+    __shared__ InstMeta sm;
+    __shared__ uint32_t tab[FILTER_MAX_CELLS];
+    uint64_t mn1 = ~0ull, mx1 = 0, mnR = ~0ull, mxR = 0;      // order-preserving unsigned images of int64
+    for (int p = tid; p < n; p += nt) {
+        const uint64_t e1 = (uint64_t)ldg64(inst + (size_t)p * R) ^ (1ull << 63);
+        const uint64_t eR = (uint64_t)ldg64(inst + (size_t)p * R + R - 1) ^ (1ull << 63);
         mn1 = min(mn1, e1); mx1 = max(mx1, e1);
         mnR = min(mnR, eR); mxR = max(mxR, eR);
     }
-    __shared__ int64_t s[4][8];
-    mn1 = (int64_t)warp_reduce((uint64_t)mn1 ^ (1ull << 63), OpMin()) ;   // order-preserving map to unsigned
-    mx1 = (int64_t)warp_reduce((uint64_t)mx1 ^ (1ull << 63), OpMax());
-    mnR = (int64_t)warp_reduce((uint64_t)mnR ^ (1ull << 63), OpMin());
-    mxR = (int64_t)warp_reduce((uint64_t)mxR ^ (1ull << 63), OpMax());
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    mn1 = warp_reduce(mn1, OpMin()); mx1 = warp_reduce(mx1, OpMax());
+    mnR = warp_reduce(mnR, OpMin()); mxR = warp_reduce(mxR, OpMax());
     if (lane == 0) { s[0][warp] = mn1; s[1][warp] = mx1; s[2][warp] = mnR; s[3][warp] = mxR; }
     __syncthreads();
-    if (threadIdx.x == 0) {
-        uint64_t a = (uint64_t)s[0][0], c = (uint64_t)s[1][0], d = (uint64_t)s[2][0], e = (uint64_t)s[3][0];
-        for (int w = 1; w < (int)(blockDim.x >> 5); ++w) {
-            a = min(a, (uint64_t)s[0][w]); c = max(c, (uint64_t)s[1][w]);
-            d = min(d, (uint64_t)s[2][w]); e = max(e, (uint64_t)s[3][w]);
-        }
+    if (tid == 0) {
+        uint64_t a = s[0][0], c = s[1][0], d = s[2][0], e = s[3][0];
+        for (int w = 1; w < nw; ++w) { a = min(a, s[0][w]); c = max(c, s[1][w]); d = min(d, s[2][w]); e = max(e, s[3][w]); }
         const int64_t tmin = (int64_t)(a ^ (1ull << 63)), t0 = (int64_t)(c ^ (1ull << 63));
         const int64_t lmin = (int64_t)(d ^ (1ull << 63)), tmax = (int64_t)(e ^ (1ull << 63));
         InstMeta m;
         m.tmin = tmin;
         m.status = ZL_OK;
+        m.sh = 0; m.ncell = 0; m.count = 0; m.pad = 0;
         if (tmin < 0 || tmax >= VALUE_LIMIT || tmax < tmin || lmin < tmin) {
             m.status = ZL_ERR_INVALID_ARG;     // outside [0, 2^62), or first/last columns out of order
             m.t0 = m.lmin = m.tend = 1; m.use32 = 1;
@@ -90,8 +114,116 @@ __global__ void __launch_bounds__(256) k_prologue(const int64_t *ts, int n, int 
             m.tend = (uint64_t)(tmax - tmin) + 1;
             m.use32 = m.tend < 0xfffffffeull;
             if (objective == ZL_OBJ_SUM && m.tend > (uint64_t)INT64_MAX / (uint64_t)n) m.status = ZL_ERR_UNSUPPORTED;
+            if (objective == ZL_OBJ_RANGE && table_all && m.use32 && m.status == ZL_OK) {
+                uint32_t sh = 0;
+                while (((m.lmin - 1) >> sh) >= (uint64_t)max_cells) ++sh;
+                m.sh = sh;
+                m.ncell = (uint32_t)((m.lmin - 1) >> sh) + 1;
+            }
         }
-        meta[b] = m;
+        sm = m;
+    }
+    __syncthreads();
+    const InstMeta M = sm;
+    if (M.ncell > 0) {
+        const uint32_t ncell = M.ncell, sh = M.sh, lmin = (uint32_t)M.lmin;
+        const int64_t tmin = M.tmin;
+        for (uint32_t c = tid; c < ncell; c += nt) tab[c] = (uint32_t)M.t0;
+        __syncthreads();
+        // one slow row per warp: the row with the longest span in the warp's group of rows
+        const int groups = min(n, FILTER_ROWS);
+        const int gsz = (n + groups - 1) / groups;
+        for (int gidx = warp; gidx < groups; gidx += nw) {
+            const int p0 = gidx * gsz, p1 = min(p0 + gsz, n);
+            uint64_t best = 0;                                   // (span << 20) | (row - p0) needs span < 2^44: use two steps
+            int bestp = -1;
+            uint64_t bspan = 0;
+            for (int p = p0 + lane; p < p1; p += 32) {
+                const uint64_t span = (uint64_t)(ldg64(inst + (size_t)p * R + R - 1) - ldg64(inst + (size_t)p * R));
+                if (bestp < 0 || span > bspan) { bspan = span; bestp = p; }
+            }
+            best = warp_reduce(bspan, OpMax());
+            const unsigned who = __ballot_sync(FULL, bestp >= 0 && bspan == best);
+            if (!who) continue;
+            const int row = __shfl_sync(FULL, bestp, __ffs(who) - 1);
+            const int64_t *rp = inst + (size_t)row * R;
+            // element i is the first element at or after every cell start in (e_{i-1}, e_i]
+            for (int i0 = 1; i0 < R; i0 += 32) {
+                const int i = i0 + lane;
+                uint32_t prev = 0xffffffffu, curv = 0;
+                if (i < R) {
+                    prev = (uint32_t)(ldg64(rp + i - 1) - tmin + 1);
+                    curv = (uint32_t)(ldg64(rp + i) - tmin + 1);
+                }
+                if (i < R && prev <= lmin) {
+                    // cell starts are 1 + (c << sh); cells with prev < start <= curv
+                    uint32_t c_from = ((prev - 1) >> sh) + 1;
+                    uint32_t c_to = min((curv - 1) >> sh, ncell - 1);
+                    for (uint32_t c = c_from; c <= c_to && c < ncell; ++c) atomicMax(&tab[c], curv);
+                }
+                const uint32_t first_prev = __shfl_sync(FULL, prev, 0);
+                if (first_prev > lmin) break;                     // the rest of the row lies after lmin
+            }
+        }
+        __syncthreads();
+        uint32_t *tg = table_all + (size_t)b * max_cells;
+        for (uint32_t c = tid; c < ncell; c += nt) tg[c] = tab[c];
+    }
+    if (tid == 0) meta[b] = M;
+    (void)flags;
+}
+
+// ------------------------------------------------------------------------------ filter pass (RANGE)
+// One warp per row streams the row in storage order (coalesced 256-byte chunks), keeps the elements
+// that pass the table test and appends them, as (T << 32 | next), to the instance's list.
+__global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R, int flags, int rows_per_cta,
+                                                  InstMeta *meta, const uint32_t *table_all, int max_cells,
+                                                  uint64_t *list_all, uint32_t listcap) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    uint32_t *tab = (uint32_t *)smem;
+    const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+    const InstMeta M = meta[b];
+    if (M.status != ZL_OK || M.ncell == 0) return;
+    const uint32_t ncell = M.ncell, sh = M.sh, lmin = (uint32_t)M.lmin;
+    const int64_t tmin = M.tmin;
+    const uint32_t *tg = table_all + (size_t)b * max_cells;
+    for (uint32_t c = tid; c < ncell; c += nt) tab[c] = tg[c];
+    __syncthreads();
+    const bool full = (flags & ZL_FLAG_FULL_SWEEP) != 0;
+    uint64_t *list = list_all + (size_t)b * listcap;
+    unsigned int *counter = &meta[b].count;
+    const int r0 = blockIdx.x * rows_per_cta, r1 = min(r0 + rows_per_cta, n);
+    for (int r = r0 + warp; r < r1; r += nw) {
+        if (*(volatile unsigned int *)counter > listcap) break;    // the list overflowed: this instance takes the general path
+        const int64_t *row = ts + ((size_t)b * n + r) * R;
+        uint32_t curT = lane < R ? (uint32_t)(ldg64(row + lane) - tmin + 1) : 0xffffffffu;
+        for (int i0 = 0; i0 < R; i0 += 32) {
+            const int inext = i0 + 32 + lane;
+            const uint32_t nxtT = inext < R ? (uint32_t)(ldg64(row + inext) - tmin + 1) : 0xffffffffu;
+            const uint32_t T = curT;
+            uint32_t nx = __shfl_down_sync(FULL, T, 1);
+            const uint32_t nfirst = __shfl_sync(FULL, nxtT, 0);
+            if (lane == 31) nx = nfirst;                            // 0xffffffff past the end of the row
+            const bool valid = i0 + lane < R && T <= lmin;
+            bool keep = false;
+            if (valid) {
+                const uint32_t L = tab[(T - 1) >> sh];
+                keep = nx > max(T, L);
+            }
+            const unsigned km = __ballot_sync(FULL, keep);
+            if (km) {
+                unsigned base = 0;
+                const int leader = __ffs(km) - 1;
+                if (lane == leader) base = atomicAdd(counter, __popc(km));
+                base = __shfl_sync(FULL, base, leader);
+                if (keep) {
+                    const unsigned pos = base + __popc(km & ((1u << lane) - 1u));
+                    if (pos < listcap) list[pos] = ((uint64_t)T << 32) | nx;
+                }
+            }
+            if (!full && __shfl_sync(FULL, T, 31) > lmin) break;   // rows are sorted: nothing later is <= lmin
+            curT = nxtT;
+        }
     }
 }
 
@@ -155,6 +287,34 @@ __device__ void run_batch(Key<K> *keys, int m, K t0, int n, uint64_t *tmp64, K c
         carryC += totc;
     }
     __syncthreads();
+}
+
+// Block minimum of (objective, time) over the per-thread bests -> out.  red: 32 shared words.
+__device__ void block_best_to_result(uint64_t bd, uint64_t bt, uint32_t status, uint64_t *red, unsigned int *sstatus,
+                                     SegResult &out) {
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+    for (int d = 16; d > 0; d >>= 1) {
+        const uint64_t od = shfl_xor(bd, d), ot = shfl_xor(bt, d);
+        if (od < bd || (od == bd && ot < bt)) { bd = od; bt = ot; }
+    }
+    __syncthreads();
+    if (lane == 0) red[tid >> 5] = bd;
+    __syncthreads();
+    // two steps: the minimum objective, then the minimum time among its holders
+    uint64_t gd = ~0ull;
+    for (int w = 0; w < (nt >> 5); ++w) gd = min(gd, red[w]);
+    __syncthreads();
+    if (lane == 0) red[tid >> 5] = bd == gd ? bt : ~0ull;
+    __syncthreads();
+    uint64_t gt = ~0ull;
+    for (int w = 0; w < (nt >> 5); ++w) gt = min(gt, red[w]);
+    if (status != ZL_OK) atomicMax(sstatus, status);
+    __syncthreads();
+    if (tid == 0) {
+        out.d = gd; out.t = gt;
+        out.valid = gd != ~0ull || gt != ~0ull;
+        out.status = (int32_t)*sstatus;
+    }
 }
 
 // ------------------------------------------------------------------------------ sweep
@@ -352,30 +512,7 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
             run_batch<K, OBJ>(keys, (int)count_before, t0, n, sh.tmp, carryMax, carryS, carryC, bd, bt);
     }
 
-    // ---- block minimum of (objective, time)
-    for (int d = 16; d > 0; d >>= 1) {
-        const uint64_t od = shfl_xor(bd, d), ot = shfl_xor(bt, d);
-        if (od < bd || (od == bd && ot < bt)) { bd = od; bt = ot; }
-    }
-    __syncthreads();
-    uint64_t *red = sh.tmp;
-    if (lane == 0) { red[(tid >> 5)] = bd; }
-    __syncthreads();
-    // two-step: first the minimum objective, then the minimum time among its holders
-    uint64_t gd = ~0ull;
-    for (int w = 0; w < (nt >> 5); ++w) gd = min(gd, red[w]);
-    __syncthreads();
-    if (lane == 0) red[(tid >> 5)] = bd == gd ? bt : ~0ull;
-    __syncthreads();
-    uint64_t gt = ~0ull;
-    for (int w = 0; w < (nt >> 5); ++w) gt = min(gt, red[w]);
-    if (status != ZL_OK) atomicMax(&sh.status, status);
-    __syncthreads();
-    if (tid == 0) {
-        out.d = gd; out.t = gt;
-        out.valid = gd != ~0ull || gt != ~0ull;
-        out.status = (int32_t)sh.status;
-    }
+    block_best_to_result(bd, bt, status, sh.tmp, &sh.status, out);
 }
 
 template <int OBJ>
@@ -385,6 +522,7 @@ __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
     const int b = blockIdx.y;
     const InstMeta M = P.meta[b];
     SegResult &out = P.seg[(size_t)b * P.nseg + blockIdx.x];
+    if (handled_by_filter(M, P.listcap)) return;             // k_small wrote this instance's result
     if (M.status != ZL_OK) {
         if (threadIdx.x == 0) { out.d = ~0ull; out.t = ~0ull; out.valid = 0; out.status = ZL_OK; }
         return;
@@ -402,9 +540,30 @@ __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
     }
 }
 
+// Sort and sweep the filtered list of an instance in one CTA.
+__global__ void __launch_bounds__(1024) k_small(InstMeta *meta, const uint64_t *list_all, uint32_t listcap, int n,
+                                                int nseg, SegResult *seg) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ uint64_t tmp[34];
+    __shared__ unsigned int sstatus;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const InstMeta M = meta[b];
+    if (M.status != ZL_OK || !handled_by_filter(M, listcap)) return;
+    Key<uint32_t> *keys = (Key<uint32_t> *)smem;
+    const uint64_t *list = list_all + (size_t)b * listcap;
+    const int m = (int)M.count;
+    for (int i = tid; i < m; i += blockDim.x) keys[i].w = list[i];
+    if (tid == 0) sstatus = 0;
+    __syncthreads();
+    uint64_t bd = ~0ull, bt = ~0ull, cs = 0;
+    uint32_t cc = 0;
+    run_batch<uint32_t, ZL_OBJ_RANGE>(keys, m, (uint32_t)M.t0, n, tmp, (uint32_t)0, cs, cc, bd, bt);
+    block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nseg]);
+}
+
 // ------------------------------------------------------------------------------ finalize
 __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int R, int nseg, int objective,
-                                                  const InstMeta *meta, const SegResult *seg,
+                                                  uint32_t listcap, const InstMeta *meta, const SegResult *seg,
                                                   int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
     const int b = blockIdx.x;
     const InstMeta M = meta[b];
@@ -415,7 +574,8 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
         uint64_t bd = ~0ull, bt = ~0ull;
         bool have = false;
         if (st == ZL_OK) {
-            for (int s = 0; s < nseg; ++s) {
+            const int nseg_used = handled_by_filter(M, listcap) ? 1 : nseg;
+            for (int s = 0; s < nseg_used; ++s) {
                 const SegResult r = seg[(size_t)b * nseg + s];
                 if (r.status != ZL_OK) st = max(st, r.status);
                 if (!r.valid) continue;
@@ -540,16 +700,19 @@ struct zl_handle {
     int num_sms;
     zl::InstMeta *d_meta;
     zl::SegResult *d_seg;
+    uint32_t *d_table;       // RANGE: filter tables, [max_batch][max_cells]
+    uint64_t *d_list;        // RANGE: filtered (T, next) lists, [max_batch][listcap]
+    int max_cells, listcap;
     size_t ws_bytes;
     // host-buffer path
     int64_t *s_ts; int32_t *s_idx; int64_t *s_barrier; int64_t *s_wait; int32_t *s_status;
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter;
     int last_cuda_error;
     int launches;
-    // optional per-kernel timing: 4 events per recorded call
+    // optional per-kernel timing: PROF_EVENTS events per recorded call
     cudaEvent_t *prof_ev;
     int prof_cap, prof_calls;
 };
@@ -560,6 +723,59 @@ int pow2_floor(int x) { int p = 1; while (p * 2 <= x) p *= 2; return p; }
 int pow2_ceil(int x) { int p = 1; while (p < x) p *= 2; return p; }
 
 struct LaunchPlan { int threads, G, nseg, cap, target; size_t smem; };
+constexpr int PROF_EVENTS = 5;
+
+// Everything one call enqueues, for both the handle-based and the fixed-scratch entry points.
+struct Pipeline {
+    const int64_t *ts; int B, n, R, objective, flags, num_sms;
+    zl::InstMeta *meta; zl::SegResult *seg;
+    uint32_t *table; uint64_t *list; int max_cells, listcap;      // table == nullptr: no filter path
+    int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;
+};
+
+void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_t *ev) {
+    const bool filter = q.table != nullptr && q.objective == ZL_OBJ_RANGE;
+    const uint32_t listcap = filter ? (uint32_t)q.listcap : 0u;
+    if (ev) cudaEventRecord(ev[0], st);
+    zl::k_prologue<<<q.B, 1024, 0, st>>>(q.ts, q.n, q.R, q.objective, q.flags, q.meta, filter ? q.table : nullptr, q.max_cells);
+    if (q.flags & ZL_FLAG_CHECK_SORTED) {
+        const size_t total = (size_t)q.B * q.n * q.R;
+        const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)q.num_sms * 16);
+        zl::k_check_sorted<<<blocks, 256, 0, st>>>(q.ts, q.n, q.R, total, q.meta);
+    }
+    if (ev) cudaEventRecord(ev[1], st);
+    if (filter) {
+        const int threads = std::max(64, std::min(1024, 32 * pow2_ceil(std::min(q.n, 32))));
+        const int nw = threads / 32;
+        long long rpc = ((long long)q.n * q.B / (4LL * q.num_sms) + nw - 1) / nw * nw;
+        rpc = std::max<long long>(nw, std::min<long long>(rpc, (q.n + nw - 1) / nw * nw));
+        const dim3 grid((unsigned)((q.n + rpc - 1) / rpc), q.B);
+        zl::k_filter<<<grid, threads, (size_t)q.max_cells * 4, st>>>(q.ts, q.n, q.R, q.flags, (int)rpc, q.meta, q.table,
+                                                                   q.max_cells, q.list, listcap);
+    }
+    if (ev) cudaEventRecord(ev[2], st);
+    if (filter) {
+        const int threads = std::max(128, std::min(1024, q.listcap / 4));
+        zl::k_small<<<q.B, threads, (size_t)q.listcap * 8, st>>>(q.meta, q.list, listcap, q.n, p.nseg, q.seg);
+    }
+    zl::SweepParams sp;
+    sp.ts = q.ts; sp.meta = q.meta; sp.seg = q.seg;
+    sp.n = q.n; sp.R = q.R; sp.nseg = p.nseg; sp.G = p.G; sp.cap = p.cap; sp.flags = q.flags; sp.target = p.target;
+    sp.listcap = listcap;
+    const dim3 grid(p.nseg, q.B);
+    if (q.objective == ZL_OBJ_RANGE) zl::k_sweep<ZL_OBJ_RANGE><<<grid, p.threads, p.smem, st>>>(sp);
+    else zl::k_sweep<ZL_OBJ_SUM><<<grid, p.threads, p.smem, st>>>(sp);
+    if (ev) cudaEventRecord(ev[3], st);
+    zl::k_finalize<<<q.B, 256, 0, st>>>(q.ts, q.n, q.R, p.nseg, q.objective, listcap, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
+    if (ev) cudaEventRecord(ev[4], st);
+}
+
+cudaError_t raise_shared_memory_limits() {
+    cudaError_t e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_small, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    return e;
+}
 
 LaunchPlan make_plan(const zl_handle *h, int B) {
     const int n = h->cfg.n_workers, R = h->cfg.lookahead_R;
@@ -640,18 +856,24 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     const size_t seg_b = (size_t)cfg->max_batch * zl::MAX_SEGMENTS * sizeof(zl::SegResult);
     if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_meta, meta_b);
     if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_seg, seg_b);
-    if (e == cudaSuccess) {
-        // the sweep may need more than the default 48 KB of dynamic shared memory
-        e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    size_t table_b = 0, list_b = 0;
+    if (cfg->objective == ZL_OBJ_RANGE) {
+        const long long N = (long long)cfg->n_workers * cfg->lookahead_R;
+        h->max_cells = std::max(64, std::min(zl::FILTER_MAX_CELLS, pow2_ceil((int)std::min<long long>(4LL * cfg->lookahead_R, 1 << 20))));
+        h->listcap = std::max(64, std::min(16384, pow2_ceil((int)std::min<long long>(N, 1 << 20))));
+        table_b = (size_t)cfg->max_batch * h->max_cells * sizeof(uint32_t);
+        list_b = (size_t)cfg->max_batch * h->listcap * sizeof(uint64_t);
+        if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_table, table_b);
+        if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_list, list_b);
     }
+    if (e == cudaSuccess) e = raise_shared_memory_limits();   // more than the default 48 KB of dynamic shared memory
     if (e != cudaSuccess) {
         zl_status st = cuda_fail(nullptr, e);
-        cudaFree(h->d_meta); cudaFree(h->d_seg);
+        cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_table); cudaFree(h->d_list);
         delete h;
         return st;
     }
-    h->ws_bytes = meta_b + seg_b;
+    h->ws_bytes = meta_b + seg_b + table_b + list_b;
     *out = h;
     return ZL_OK;
 }
@@ -659,7 +881,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
 zl_status zl_profile_end(zl_handle *h) {
     if (!h) return ZL_ERR_INVALID_ARG;
     if (h->prof_ev) {
-        for (int i = 0; i < 4 * h->prof_cap; ++i) cudaEventDestroy(h->prof_ev[i]);
+        for (int i = 0; i < PROF_EVENTS * h->prof_cap; ++i) cudaEventDestroy(h->prof_ev[i]);
         delete[] h->prof_ev;
     }
     h->prof_ev = nullptr;
@@ -671,9 +893,9 @@ zl_status zl_profile_begin(zl_handle *h, int32_t max_calls) {
     if (!h || max_calls < 1 || max_calls > 65536) return ZL_ERR_INVALID_ARG;
     zl_profile_end(h);
     ZL_CUDA(h, cudaSetDevice(h->cfg.device));
-    h->prof_ev = new (std::nothrow) cudaEvent_t[4 * (size_t)max_calls];
+    h->prof_ev = new (std::nothrow) cudaEvent_t[PROF_EVENTS * (size_t)max_calls];
     if (!h->prof_ev) return ZL_ERR_NOMEM;
-    for (int i = 0; i < 4 * max_calls; ++i) {
+    for (int i = 0; i < PROF_EVENTS * max_calls; ++i) {
         cudaError_t e = cudaEventCreate(&h->prof_ev[i]);
         if (e != cudaSuccess) {
             for (int j = 0; j < i; ++j) cudaEventDestroy(h->prof_ev[j]);
@@ -687,18 +909,18 @@ zl_status zl_profile_begin(zl_handle *h, int32_t max_calls) {
     return ZL_OK;
 }
 
-zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_prologue, float *ms_sweep, float *ms_finalize) {
-    if (!h || !calls || !ms_prologue || !ms_sweep || !ms_finalize) return ZL_ERR_INVALID_ARG;
+zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_stage) {
+    if (!h || !calls || !ms_stage) return ZL_ERR_INVALID_ARG;
     *calls = h->prof_calls;
-    *ms_prologue = *ms_sweep = *ms_finalize = 0.f;
+    for (int k = 0; k < PROF_EVENTS - 1; ++k) ms_stage[k] = 0.f;
     for (int c = 0; c < h->prof_calls; ++c) {
-        cudaEvent_t *ev = h->prof_ev + 4 * (size_t)c;
-        ZL_CUDA(h, cudaEventSynchronize(ev[3]));
-        float a = 0.f, b = 0.f, d = 0.f;
-        ZL_CUDA(h, cudaEventElapsedTime(&a, ev[0], ev[1]));
-        ZL_CUDA(h, cudaEventElapsedTime(&b, ev[1], ev[2]));
-        ZL_CUDA(h, cudaEventElapsedTime(&d, ev[2], ev[3]));
-        *ms_prologue += a; *ms_sweep += b; *ms_finalize += d;
+        cudaEvent_t *ev = h->prof_ev + PROF_EVENTS * (size_t)c;
+        ZL_CUDA(h, cudaEventSynchronize(ev[PROF_EVENTS - 1]));
+        for (int k = 0; k < PROF_EVENTS - 1; ++k) {
+            float ms = 0.f;
+            ZL_CUDA(h, cudaEventElapsedTime(&ms, ev[k], ev[k + 1]));
+            ms_stage[k] += ms;
+        }
     }
     h->prof_calls = 0;
     return ZL_OK;
@@ -707,7 +929,7 @@ zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_prologue, floa
 zl_status zl_destroy(zl_handle *h) {
     if (!h) return ZL_OK;
     cudaSetDevice(h->cfg.device);
-    cudaFree(h->d_meta); cudaFree(h->d_seg);
+    cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_table); cudaFree(h->d_list);
     cudaFree(h->s_ts); cudaFree(h->s_idx); cudaFree(h->s_barrier); cudaFree(h->s_wait); cudaFree(h->s_status);
     if (h->s_stream) cudaStreamDestroy(h->s_stream);
     zl_profile_end(h);
@@ -727,6 +949,8 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
     } else if (!strcmp(key, "segments")) {
         if (value > zl::MAX_SEGMENTS) return ZL_ERR_INVALID_ARG;
         h->opt_segments = value;
+    } else if (!strcmp(key, "no_filter")) {
+        h->opt_no_filter = value != 0;
     } else if (!strcmp(key, "round_factor")) {
         if (value > 100000) return ZL_ERR_INVALID_ARG;
         h->opt_round_factor = value;
@@ -737,7 +961,11 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
 }
 
 size_t zl_workspace_bytes(const zl_handle *h) { return h ? h->ws_bytes + h->staging_bytes : 0; }
-int32_t zl_launches_per_call(const zl_handle *h) { return h ? 3 + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0) : 0; }
+int32_t zl_launches_per_call(const zl_handle *h) {
+    if (!h) return 0;
+    const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter;
+    return 3 + (filter ? 2 : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
+}
 int32_t zl_segments_per_instance(const zl_handle *h, int32_t B) { return h && B >= 1 ? make_plan(h, B).nseg : 0; }
 int32_t zl_last_cuda_error(const zl_handle *h) { return h ? h->last_cuda_error : 0; }
 
@@ -753,24 +981,14 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     const LaunchPlan p = make_plan(h, B);
     if (p.smem > 200 * 1024) return ZL_ERR_UNSUPPORTED;
 
-    cudaEvent_t *ev = (h->prof_ev && h->prof_calls < h->prof_cap) ? h->prof_ev + 4 * (size_t)h->prof_calls : nullptr;
-    if (ev) cudaEventRecord(ev[0], st);
-    zl::k_prologue<<<B, 256, 0, st>>>(d_ts, n, R, obj, h->d_meta);
-    if (h->cfg.flags & ZL_FLAG_CHECK_SORTED) {
-        const size_t total = (size_t)B * n * R;
-        const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)h->num_sms * 16);
-        zl::k_check_sorted<<<blocks, 256, 0, st>>>(d_ts, n, R, total, h->d_meta);
-    }
-    zl::SweepParams sp;
-    sp.ts = d_ts; sp.meta = h->d_meta; sp.seg = h->d_seg;
-    sp.n = n; sp.R = R; sp.nseg = p.nseg; sp.G = p.G; sp.cap = p.cap; sp.flags = h->cfg.flags; sp.target = p.target;
-    const dim3 grid(p.nseg, B);
-    if (ev) cudaEventRecord(ev[1], st);
-    if (obj == ZL_OBJ_RANGE) zl::k_sweep<ZL_OBJ_RANGE><<<grid, p.threads, p.smem, st>>>(sp);
-    else zl::k_sweep<ZL_OBJ_SUM><<<grid, p.threads, p.smem, st>>>(sp);
-    if (ev) cudaEventRecord(ev[2], st);
-    zl::k_finalize<<<B, 256, 0, st>>>(d_ts, n, R, p.nseg, obj, h->d_meta, h->d_seg, d_idx, d_barrier, d_wait, d_status);
-    if (ev) { cudaEventRecord(ev[3], st); ++h->prof_calls; }
+    cudaEvent_t *ev = (h->prof_ev && h->prof_calls < h->prof_cap) ? h->prof_ev + PROF_EVENTS * (size_t)h->prof_calls : nullptr;
+    Pipeline q;
+    q.ts = d_ts; q.B = B; q.n = n; q.R = R; q.objective = obj; q.flags = h->cfg.flags; q.num_sms = h->num_sms;
+    q.meta = h->d_meta; q.seg = h->d_seg;
+    q.table = h->opt_no_filter ? nullptr : h->d_table; q.list = h->d_list; q.max_cells = h->max_cells; q.listcap = h->listcap;
+    q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
+    enqueue(q, p, st, ev);
+    if (ev) ++h->prof_calls;
     ZL_CUDA(h, cudaGetLastError());
     h->launches += zl_launches_per_call(h);
     return ZL_OK;
@@ -872,8 +1090,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
             void *ptr = nullptr;
             cudaError_t e = cudaGetSymbolAddress((void **)&ptr, g_noalloc_scratch);
             if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_noalloc_sms[dev], cudaDevAttrMultiProcessorCount, dev);
-            if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e == cudaSuccess) e = raise_shared_memory_limits();
             if (e != cudaSuccess || !ptr) return ZL_ERR_CUDA;
             g_noalloc_ptr[dev] = ptr;
         }
@@ -888,23 +1105,15 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     }
     zl::InstMeta *meta = (zl::InstMeta *)g_noalloc_ptr[dev];
     zl::SegResult *seg = (zl::SegResult *)((unsigned char *)g_noalloc_ptr[dev] + NOALLOC_META_BYTES);
-    cudaStream_t st = (cudaStream_t)cuda_stream;
     // Nothing in the scratch has to start at zero: the prologue rewrites every InstMeta of this call and
     // every sweep CTA rewrites its SegResult before finalize reads them, so the last call's contents are
-    // never read.
-    zl::k_prologue<<<B, 256, 0, st>>>(d_ts, n_workers, lookahead_R, objective, meta);
-    if (flags & ZL_FLAG_CHECK_SORTED) {
-        const size_t total = (size_t)B * n_workers * lookahead_R;
-        const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)tmp.num_sms * 16);
-        zl::k_check_sorted<<<blocks, 256, 0, st>>>(d_ts, n_workers, lookahead_R, total, meta);
-    }
-    zl::SweepParams sp;
-    sp.ts = d_ts; sp.meta = meta; sp.seg = seg;
-    sp.n = n_workers; sp.R = lookahead_R; sp.nseg = p.nseg; sp.G = p.G; sp.cap = p.cap; sp.flags = flags; sp.target = p.target;
-    const dim3 grid(p.nseg, B);
-    if (objective == ZL_OBJ_RANGE) zl::k_sweep<ZL_OBJ_RANGE><<<grid, p.threads, p.smem, st>>>(sp);
-    else zl::k_sweep<ZL_OBJ_SUM><<<grid, p.threads, p.smem, st>>>(sp);
-    zl::k_finalize<<<B, 256, 0, st>>>(d_ts, n_workers, lookahead_R, p.nseg, objective, meta, seg, d_idx, d_barrier, d_wait, d_status);
+    // never read.  (The filter path of the handle-based entry point needs two more buffers and is not used here.)
+    Pipeline q;
+    q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
+    q.meta = meta; q.seg = seg;
+    q.table = nullptr; q.list = nullptr; q.max_cells = 0; q.listcap = 0;
+    q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
+    enqueue(q, p, (cudaStream_t)cuda_stream, nullptr);
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;
 }
 

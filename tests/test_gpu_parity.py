@@ -21,10 +21,20 @@ def gpu_select(ts_np, objective, flags=0, options=None):
     h = zl.ZipLine(n, R, B, objective, 0, flags)
     for k, v in (options or {}).items():
         h.set_option(k, v)
-    sel = h.select_batched(torch.from_numpy(ts_np).cuda())
+    d_ts = torch.from_numpy(ts_np).cuda()
+    sel = h.select_batched(d_ts)
     torch.cuda.synchronize()
+    got = (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy())
+    if objective == 0 and "no_filter" not in (options or {}):
+        # RANGE has two routes (filter pass + one sort, or the segment sweep): both must agree exactly
+        h.set_option("no_filter", 1)
+        sel2 = h.select_batched(d_ts)
+        torch.cuda.synchronize()
+        for a, b in zip(got, (sel2.idx.cpu().numpy(), sel2.barrier.cpu().numpy(), sel2.wait.cpu().numpy(),
+                              sel2.status.cpu().numpy())):
+            assert (a == b).all(), "filter route and segment-sweep route disagree"
     h.destroy()
-    return sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()
+    return got
 
 
 def assert_same(ts_np, objective, got, fn=None, which=None):
@@ -185,7 +195,7 @@ def test_host_detected_errors():
         h.select_batched(ts)             # B > max_batch
     with pytest.raises(zl.ZipLineError):
         h.set_option("no_such_option", 1)
-    assert h.launches_per_call == 3 and h.workspace_bytes > 0
+    assert h.launches_per_call == 5 and h.workspace_bytes > 0
     h.destroy()
 
 
