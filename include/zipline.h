@@ -181,6 +181,15 @@ size_t   zl_noalloc_scratch_bytes(void);   /* size of the fixed device array it 
 /* Free the scratch and the handle.  NULL is a no-op. */
 zl_status zl_destroy(zl_handle *h);
 
+/*
+ * Diagnostic (no counterpart in the paper): for the last zl_select_batched on h and each of
+ * its first B instances, how many elements passed the RANGE filter pass (h_filtered), how many of
+ * those passed the refinement (h_refined), and whether a survivor list overflowed, in which case
+ * the segment sweep handled the instance instead (h_overflow).  Host arrays of B uint32, any of
+ * which may be NULL.  Synchronises the device.
+ */
+zl_status zl_filter_counts(zl_handle *h, int32_t B, uint32_t *h_filtered, uint32_t *h_refined, uint32_t *h_overflow);
+
 /* Tuning knobs of a handle (host side; take effect at the next call).
  * key: "threads" (128..1024, power of two), "lanes_per_row" (1..32, power of two),
  * "segments" (time segments per instance, >= 1), "round_factor" (percent of the

@@ -22,7 +22,7 @@ EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace
            "zl_set_option", "zl_status_string", "zl_workspace_bytes", "zl_launches_per_call",
            "zl_segments_per_instance", "zl_max_workers", "zl_trace_max_elements", "zl_last_cuda_error",
            "zl_profile_begin", "zl_profile_read", "zl_profile_end",
-           "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes")
+           "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes", "zl_filter_counts")
 
 
 class zl_config(ctypes.Structure):
@@ -49,6 +49,8 @@ def _load() -> ctypes.CDLL:
     lib.zl_profile_begin.argtypes = [vp, i32]
     lib.zl_profile_read.argtypes = [vp, vp, vp]
     lib.zl_profile_end.argtypes = [vp]
+    lib.zl_filter_counts.argtypes = [vp, i32, vp, vp, vp]
+    lib.zl_filter_counts.restype = ctypes.c_int
     lib.zl_select_batched_noalloc.argtypes = [i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
     lib.zl_select_batched_noalloc.restype = ctypes.c_int
     lib.zl_noalloc_max_batch.restype = ctypes.c_int
@@ -161,6 +163,13 @@ class ZipLine:
 
     def profile_end(self):
         _check(lib.zl_profile_end(self._h), "zl_profile_end")
+
+    def filter_counts(self, B: int):
+        """(filter-pass survivors, refined survivors, overflow flags) per instance of the last call.  Synchronises."""
+        f, r, o = (ctypes.c_uint32 * B)(), (ctypes.c_uint32 * B)(), (ctypes.c_uint32 * B)()
+        _check(lib.zl_filter_counts(self._h, B, ctypes.addressof(f), ctypes.addressof(r), ctypes.addressof(o)),
+               "zl_filter_counts")
+        return list(f), list(r), list(o)
 
     def set_option(self, key: str, value: int):
         _check(lib.zl_set_option(self._h, key.encode(), int(value)), f"zl_set_option({key})")

@@ -12,6 +12,7 @@
 //              are independent.
 //   finalize   minimum over the segments of an instance, barrier, per-worker index recovery.
 #include <cuda_runtime.h>
+#include <stddef.h>
 #include <stdint.h>
 #include <stdio.h>
 #include <string.h>
@@ -36,10 +37,11 @@ struct InstMeta {
     uint64_t tend;       // max_p e^p_R, relative  (= span + 1)
     int32_t status;      // zl_status of the instance
     int32_t use32;       // relative times fit 32 bits
-    uint32_t sh;         // filter table: cell c covers relative times [1 + (c << sh), 1 + ((c + 1) << sh))
-    uint32_t ncell;      // cells in use (0: the instance does not take the filter path)
-    uint32_t count;      // survivors appended by the filter pass (may run past the list capacity)
-    uint32_t pad;
+    uint32_t cscale;     // filter route: time cell of relative time T = ((T - 1) * cscale) >> 32 (monotone in T);
+                         // 0: the instance does not take the filter route
+    uint32_t count;      // survivors of the filter pass
+    uint32_t count2;     // survivors of the refinement
+    uint32_t overflow;   // a survivor list overflowed: the instance takes the segment sweep instead
 };
 
 struct SegResult {
@@ -49,18 +51,42 @@ struct SegResult {
     int32_t status;
 };
 
+// Buffers of the RANGE filter route (all nullptr / 0 when the route is off).  Time is cut into
+// `cells` cells per instance; `nbk` buckets are runs of cells / nbk consecutive cells.
+struct FilterBufs {
+    uint32_t *table;     // [B][cells]        lower bound of G at the start of each cell (from a few slow rows)
+    uint32_t *rowhint;   // [B][n]            estimated number of elements of a row that are <= lmin
+    uint32_t *cellmax;   // [B][cells]        max `next` over the filter pass's survivors of each cell
+    uint32_t *rcnt;      // [B][nreg]         survivors per region (one region per CTA of the filter pass)
+    uint64_t *list1;     // [B][list1cap]     survivors of the filter pass as (T << 32 | next), by region
+    uint32_t *bcnt;      // [B][nbk]          survivors of the refinement per bucket
+    uint64_t *list2;     // [B][nbk][capb]    survivors of the refinement
+    int32_t cells, nbk, capb, grp;           // grp: fewest buckets per CTA of the bucket sweep
+    int32_t nreg, regcap, list1cap;          // set per call: regions per instance and their capacity
+};
+
 struct SweepParams {
     const int64_t *ts;
     InstMeta *meta;
     SegResult *seg;
-    int32_t n, R, nseg, G, cap, flags, target;
-    uint32_t listcap;    // > 0: instances whose filtered list fits are handled by k_small, not here
+    int32_t n, R, B, nseg, nres, G, cap, flags, target;   // nres: SegResult slots per instance
+    int32_t filter;      // instances handled by the filter route are skipped
 };
 
-// An instance goes through the filter + small-sort path when it has a table and its survivors fit the list.
-__device__ __forceinline__ bool handled_by_filter(const InstMeta &M, uint32_t listcap) {
-    return listcap > 0 && M.ncell > 0 && M.count <= listcap;
+// Buckets per CTA of the bucket sweep for an instance with `count` refined survivors: the static
+// minimum `grp`, widened (by powers of two) so that a CTA expects about a quarter batch of survivors.
+__device__ __forceinline__ int bucket_group(const FilterBufs &F, uint32_t count) {
+    int g = F.grp;
+    while (g < F.nbk && (uint64_t)count * (uint64_t)g * 2 < (uint64_t)F.nbk * (uint64_t)(F.capb / 2)) g <<= 1;
+    return g;
 }
+
+// An instance goes through the filter route when it has a table and no survivor list overflowed.
+__device__ __forceinline__ bool handled_by_filter(const InstMeta &M, int filter) {
+    return filter && M.cscale != 0 && M.overflow == 0;
+}
+
+__device__ __forceinline__ uint32_t cell_of(uint32_t T, uint32_t cscale) { return __umulhi(T - 1, cscale); }
 
 // ------------------------------------------------------------------------------ prologue
 // Column scans per instance, and (RANGE, 32-bit instances) the filter table.
@@ -79,7 +105,7 @@ constexpr int FILTER_ROWS = 32;      // rows that build the table
 constexpr int FILTER_MAX_CELLS = 8192;
 
 __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int R, int objective, int flags,
-                                                    InstMeta *meta, uint32_t *table_all, int max_cells) {
+                                                    InstMeta *meta, FilterBufs F) {
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
     const int64_t *inst = ts + (size_t)b * n * R;
     __shared__ uint64_t s[4][32];
@@ -104,7 +130,7 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
         InstMeta m;
         m.tmin = tmin;
         m.status = ZL_OK;
-        m.sh = 0; m.ncell = 0; m.count = 0; m.pad = 0;
+        m.cscale = 0; m.count = 0; m.count2 = 0; m.overflow = 0;
         if (tmin < 0 || tmax >= VALUE_LIMIT || tmax < tmin || lmin < tmin) {
             m.status = ZL_ERR_INVALID_ARG;     // outside [0, 2^62), or first/last columns out of order
             m.t0 = m.lmin = m.tend = 1; m.use32 = 1;
@@ -114,40 +140,49 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
             m.tend = (uint64_t)(tmax - tmin) + 1;
             m.use32 = m.tend < 0xfffffffeull;
             if (objective == ZL_OBJ_SUM && m.tend > (uint64_t)INT64_MAX / (uint64_t)n) m.status = ZL_ERR_UNSUPPORTED;
-            if (objective == ZL_OBJ_RANGE && table_all && m.use32 && m.status == ZL_OK) {
-                uint32_t sh = 0;
-                while (((m.lmin - 1) >> sh) >= (uint64_t)max_cells) ++sh;
-                m.sh = sh;
-                m.ncell = (uint32_t)((m.lmin - 1) >> sh) + 1;
-            }
+            if (objective == ZL_OBJ_RANGE && F.table && m.use32 && m.status == ZL_OK)
+                // (T - 1) < lmin for every T <= lmin, so ((T - 1) * cscale) >> 32 < cells
+                m.cscale = (uint32_t)max((uint64_t)1, min((uint64_t)0xffffffffu, ((uint64_t)F.cells << 32) / m.lmin));
         }
         sm = m;
     }
     __syncthreads();
     const InstMeta M = sm;
-    if (M.ncell > 0) {
-        const uint32_t ncell = M.ncell, sh = M.sh, lmin = (uint32_t)M.lmin;
+    if (M.cscale != 0) {
+        const uint32_t cells = (uint32_t)F.cells, cscale = M.cscale, lmin = (uint32_t)M.lmin;
         const int64_t tmin = M.tmin;
-        for (uint32_t c = tid; c < ncell; c += nt) tab[c] = (uint32_t)M.t0;
+        uint32_t *cmx = F.cellmax + (size_t)b * cells;
+        for (uint32_t c = tid; c < cells; c += nt) { tab[c] = (uint32_t)M.t0; cmx[c] = 0; }
+        for (int k = tid; k < F.nbk; k += nt) F.bcnt[(size_t)b * F.nbk + k] = 0;
+        // per row: how many of its elements are expected to be <= lmin (rows are close to arithmetic);
+        // the filter pass uses it only to decide how much of the row to request up front
+        for (int p = tid; p < n; p += nt) {
+            const uint64_t e1 = (uint64_t)(ldg64(inst + (size_t)p * R) - tmin) + 1;
+            const uint64_t eR = (uint64_t)(ldg64(inst + (size_t)p * R + R - 1) - tmin) + 1;
+            uint64_t est = R;
+            if (eR > e1 && (uint64_t)lmin < eR)
+                est = (uint64_t)lmin <= e1 ? 1 : ((uint64_t)lmin - e1) * (uint64_t)(R - 1) / (eR - e1) + 8;
+            F.rowhint[(size_t)b * n + p] = (uint32_t)min(est, (uint64_t)R);
+        }
         __syncthreads();
         // one slow row per warp: the row with the longest span in the warp's group of rows
         const int groups = min(n, FILTER_ROWS);
         const int gsz = (n + groups - 1) / groups;
         for (int gidx = warp; gidx < groups; gidx += nw) {
             const int p0 = gidx * gsz, p1 = min(p0 + gsz, n);
-            uint64_t best = 0;                                   // (span << 20) | (row - p0) needs span < 2^44: use two steps
             int bestp = -1;
             uint64_t bspan = 0;
             for (int p = p0 + lane; p < p1; p += 32) {
                 const uint64_t span = (uint64_t)(ldg64(inst + (size_t)p * R + R - 1) - ldg64(inst + (size_t)p * R));
                 if (bestp < 0 || span > bspan) { bspan = span; bestp = p; }
             }
-            best = warp_reduce(bspan, OpMax());
+            const uint64_t best = warp_reduce(bspan, OpMax());
             const unsigned who = __ballot_sync(FULL, bestp >= 0 && bspan == best);
             if (!who) continue;
             const int row = __shfl_sync(FULL, bestp, __ffs(who) - 1);
             const int64_t *rp = inst + (size_t)row * R;
-            // element i is the first element at or after every cell start in (e_{i-1}, e_i]
+            // element i is the first element of the row at or after every cell start in (e_{i-1}, e_i]:
+            // the cells after the one holding e_{i-1}, up to the one holding e_i
             for (int i0 = 1; i0 < R; i0 += 32) {
                 const int i = i0 + lane;
                 uint32_t prev = 0xffffffffu, curv = 0;
@@ -156,75 +191,241 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
                     curv = (uint32_t)(ldg64(rp + i) - tmin + 1);
                 }
                 if (i < R && prev <= lmin) {
-                    // cell starts are 1 + (c << sh); cells with prev < start <= curv
-                    uint32_t c_from = ((prev - 1) >> sh) + 1;
-                    uint32_t c_to = min((curv - 1) >> sh, ncell - 1);
-                    for (uint32_t c = c_from; c <= c_to && c < ncell; ++c) atomicMax(&tab[c], curv);
+                    const uint32_t c_from = cell_of(prev, cscale) + 1;
+                    const uint32_t c_to = curv <= lmin ? cell_of(curv, cscale) : cells - 1;
+                    for (uint32_t c = c_from; c <= c_to && c < cells; ++c) atomicMax(&tab[c], curv);
                 }
                 const uint32_t first_prev = __shfl_sync(FULL, prev, 0);
                 if (first_prev > lmin) break;                     // the rest of the row lies after lmin
             }
         }
         __syncthreads();
-        uint32_t *tg = table_all + (size_t)b * max_cells;
-        for (uint32_t c = tid; c < ncell; c += nt) tg[c] = tab[c];
+        uint32_t *tg = F.table + (size_t)b * cells;
+        for (uint32_t c = tid; c < cells; c += nt) tg[c] = tab[c];
     }
     if (tid == 0) meta[b] = M;
     (void)flags;
 }
 
 // ------------------------------------------------------------------------------ filter pass (RANGE)
-// One warp per row streams the row in storage order (coalesced 256-byte chunks), keeps the elements
-// that pass the table test and appends them, as (T << 32 | next), to the instance's list.
+// A CTA owns a block of rows of one instance (a "region").  Each warp streams its rows in storage
+// order through a private shared-memory ring filled by 16-byte cp.async copies (FILTER_STAGES chunks of
+// 64 timestamps in flight per warp), tests every element against the table and appends the survivors,
+// as (T << 32 | next), to the region's list; the per-cell maximum of `next` over the survivors goes to
+// cellmax for the refinement.  Rows whose length is odd, or a misaligned base, take 8-byte copies.
+constexpr int FILTER_STAGES = 4;      // ring slots per warp
+constexpr int FILTER_CHUNK = 128;     // timestamps per slot (two 16-byte copies per lane)
+constexpr int FILTER_SLOT = FILTER_CHUNK + 2;   // + the successor of the slot's last element, + padding
+
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async8(void *smem, const void *gmem) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+// wait until at most `pending` of this thread's most recent groups are still in flight
+__device__ __forceinline__ void cp_async_wait_pending(int pending) {
+    switch (pending) {
+        case 0: asm volatile("cp.async.wait_group 0;\n" ::: "memory"); break;
+        case 1: asm volatile("cp.async.wait_group 1;\n" ::: "memory"); break;
+        case 2: asm volatile("cp.async.wait_group 2;\n" ::: "memory"); break;
+        case 3: asm volatile("cp.async.wait_group 3;\n" ::: "memory"); break;
+        case 4: asm volatile("cp.async.wait_group 4;\n" ::: "memory"); break;
+        case 5: asm volatile("cp.async.wait_group 5;\n" ::: "memory"); break;
+        case 6: asm volatile("cp.async.wait_group 6;\n" ::: "memory"); break;
+        default: asm volatile("cp.async.wait_group 7;\n" ::: "memory"); break;
+    }
+}
+
+struct FilterCtx {
+    const uint32_t *tab; uint64_t *list; uint32_t *cellmax; unsigned int *scount;
+    uint32_t cscale, lmin, regcap;
+};
+
+// Table test of the (up to) two elements of a lane, warp-aggregated append of the survivors.
+__device__ __forceinline__ void filter_pair(const FilterCtx &c, int lane, bool va, uint32_t Ta, uint32_t na,
+                                            bool vb, uint32_t Tb, uint32_t nb) {
+    bool ka = false, kb = false;
+    uint32_t ca = 0, cb = 0;
+    if (va && Ta <= c.lmin) { ca = cell_of(Ta, c.cscale); ka = na > max(Ta, c.tab[ca]); }
+    if (vb && Tb <= c.lmin) { cb = cell_of(Tb, c.cscale); kb = nb > max(Tb, c.tab[cb]); }
+    const unsigned ma = __ballot_sync(FULL, ka), mb = __ballot_sync(FULL, kb);
+    if ((ma | mb) == 0) return;
+    const int na_cnt = __popc(ma), tot = na_cnt + __popc(mb);
+    unsigned base = 0;
+    if (lane == 0) base = atomicAdd(c.scount, (unsigned)tot);
+    base = __shfl_sync(FULL, base, 0);
+    const unsigned below = (1u << lane) - 1u;
+    if (ka) {
+        const unsigned pos = base + __popc(ma & below);
+        if (pos < c.regcap) c.list[pos] = ((uint64_t)Ta << 32) | na;
+        atomicMax(&c.cellmax[ca], na);
+    }
+    if (kb) {
+        const unsigned pos = base + na_cnt + __popc(mb & below);
+        if (pos < c.regcap) c.list[pos] = ((uint64_t)Tb << 32) | nb;
+        atomicMax(&c.cellmax[cb], nb);
+    }
+}
+
+// The 64 elements of a slot starting at `off`: element pairs per lane, successor of the pair from the
+// slot itself (the element after the slot's last one sits right behind it).  Returns the time of the
+// last valid element handled by lane 31 (0xffffffff past the row's end).
+__device__ __forceinline__ uint32_t filter_half(const FilterCtx &C, const int64_t *slot, int off, int i0, int R,
+                                                uint32_t tminlo, int lane) {
+    const int i = i0 + off + 2 * lane;
+    const bool va = i < R, vb = i + 1 < R;
+    const longlong2 ab = *reinterpret_cast<const longlong2 *>(slot + off + 2 * lane);
+    const uint32_t Ta = va ? (uint32_t)(uint64_t)ab.x - tminlo : 0xffffffffu;
+    const uint32_t Tb = vb ? (uint32_t)(uint64_t)ab.y - tminlo : 0xffffffffu;
+    const uint32_t nb = i + 2 < R ? (uint32_t)(uint64_t)slot[off + 2 * lane + 2] - tminlo : 0xffffffffu;
+    filter_pair(C, lane, va, Ta, Tb, vb, Tb, nb);
+    return __shfl_sync(FULL, Tb, 31);
+}
+
 __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R, int flags, int rows_per_cta,
-                                                  InstMeta *meta, const uint32_t *table_all, int max_cells,
-                                                  uint64_t *list_all, uint32_t listcap) {
+                                                  InstMeta *meta, FilterBufs F) {
     extern __shared__ __align__(16) unsigned char smem[];
-    uint32_t *tab = (uint32_t *)smem;
+    __shared__ unsigned int scount;
     const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
     const InstMeta M = meta[b];
-    if (M.status != ZL_OK || M.ncell == 0) return;
-    const uint32_t ncell = M.ncell, sh = M.sh, lmin = (uint32_t)M.lmin;
-    const int64_t tmin = M.tmin;
-    const uint32_t *tg = table_all + (size_t)b * max_cells;
-    for (uint32_t c = tid; c < ncell; c += nt) tab[c] = tg[c];
+    uint32_t *rc = F.rcnt + (size_t)b * F.nreg + blockIdx.x;
+    if (M.status != ZL_OK || M.cscale == 0) { if (tid == 0) *rc = 0; return; }
+    const uint32_t cells = (uint32_t)F.cells, lmin = (uint32_t)M.lmin;
+    const uint32_t tminlo = (uint32_t)(uint64_t)M.tmin - 1u;     // relative time = low word of t - tminlo
+    uint32_t *tab = (uint32_t *)smem;
+    int64_t *ring = (int64_t *)(smem + (size_t)cells * 4) + (size_t)warp * FILTER_STAGES * FILTER_SLOT;
+    const uint32_t *tg = F.table + (size_t)b * cells;
+    for (uint32_t c = tid; c < cells; c += nt) tab[c] = tg[c];
+    if (tid == 0) scount = 0;
     __syncthreads();
     const bool full = (flags & ZL_FLAG_FULL_SWEEP) != 0;
-    uint64_t *list = list_all + (size_t)b * listcap;
-    unsigned int *counter = &meta[b].count;
+    FilterCtx C;
+    C.tab = tab; C.list = F.list1 + (size_t)b * F.list1cap + (size_t)blockIdx.x * F.regcap;
+    C.cellmax = F.cellmax + (size_t)b * cells; C.scount = &scount;
+    C.cscale = M.cscale; C.lmin = lmin; C.regcap = (uint32_t)F.regcap;
     const int r0 = blockIdx.x * rows_per_cta, r1 = min(r0 + rows_per_cta, n);
-    for (int r = r0 + warp; r < r1; r += nw) {
-        if (*(volatile unsigned int *)counter > listcap) break;    // the list overflowed: this instance takes the general path
-        const int64_t *row = ts + ((size_t)b * n + r) * R;
-        uint32_t curT = lane < R ? (uint32_t)(ldg64(row + lane) - tmin + 1) : 0xffffffffu;
-        for (int i0 = 0; i0 < R; i0 += 32) {
-            const int inext = i0 + 32 + lane;
-            const uint32_t nxtT = inext < R ? (uint32_t)(ldg64(row + inext) - tmin + 1) : 0xffffffffu;
-            const uint32_t T = curT;
-            uint32_t nx = __shfl_down_sync(FULL, T, 1);
-            const uint32_t nfirst = __shfl_sync(FULL, nxtT, 0);
-            if (lane == 31) nx = nfirst;                            // 0xffffffff past the end of the row
-            const bool valid = i0 + lane < R && T <= lmin;
-            bool keep = false;
-            if (valid) {
-                const uint32_t L = tab[(T - 1) >> sh];
-                keep = nx > max(T, L);
-            }
-            const unsigned km = __ballot_sync(FULL, keep);
-            if (km) {
-                unsigned base = 0;
-                const int leader = __ffs(km) - 1;
-                if (lane == leader) base = atomicAdd(counter, __popc(km));
-                base = __shfl_sync(FULL, base, leader);
-                if (keep) {
-                    const unsigned pos = base + __popc(km & ((1u << lane) - 1u));
-                    if (pos < listcap) list[pos] = ((uint64_t)T << 32) | nx;
+    const bool vec2 = (R % 2 == 0) && (((uintptr_t)ts & 15) == 0);
+    const int nchunks = (R + FILTER_CHUNK - 1) / FILTER_CHUNK;
+    const size_t rstride = (size_t)nw * R;                        // between consecutive rows of this warp
+
+    // this warp's rows, in rounds of up to 32: lane j holds the request (in slots) of the round's j-th row
+    for (int rbase = r0 + warp; rbase < r1; rbase += 32 * nw) {
+        const int nrows = min(32, (r1 - rbase + nw - 1) / nw);
+        int req = 0;
+        if (lane < nrows)
+            req = full ? nchunks : min(nchunks, (int)((F.rowhint[(size_t)b * n + rbase + lane * nw] + FILTER_CHUNK - 1) / FILTER_CHUNK));
+        const int64_t *row_i = ts + ((size_t)b * n + rbase) * R, *row_p = row_i;
+        int ji = 0, ci = 0, jp = 0, cp = 0, inflight = 0, slot_i = 0, slot_p = 0;
+        int req_i = __shfl_sync(FULL, req, 0), req_p = req_i;
+        bool finished = false;                                     // the row being processed needs nothing more
+        while (jp < nrows) {
+            while (inflight < FILTER_STAGES && ji < nrows) {
+                int64_t *slot = ring + (size_t)slot_i * FILTER_SLOT;
+                const int i = ci * FILTER_CHUNK + 2 * lane;
+                if (vec2) {
+                    if (i < R) cp_async16(slot + 2 * lane, row_i + i);
+                    if (i + 64 < R) cp_async16(slot + 64 + 2 * lane, row_i + i + 64);
+                } else {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const int e = i + (k >> 1) * 64 + (k & 1);
+                        if (e < R) cp_async8(slot + (k >> 1) * 64 + 2 * lane + (k & 1), row_i + e);
+                    }
+                }
+                if (lane == 31 && i + 66 < R) cp_async8(slot + FILTER_CHUNK, row_i + i + 66);   // successor of the slot's last element
+                cp_async_commit();
+                ++inflight;
+                slot_i = slot_i + 1 == FILTER_STAGES ? 0 : slot_i + 1;
+                if (++ci == req_i) {
+                    ci = 0; ++ji; row_i += rstride;
+                    req_i = __shfl_sync(FULL, req, min(ji, 31));
                 }
             }
-            if (!full && __shfl_sync(FULL, T, 31) > lmin) break;   // rows are sorted: nothing later is <= lmin
-            curT = nxtT;
+            cp_async_wait_pending(inflight - 1);
+            __syncwarp();
+            if (!finished) {
+                const int64_t *slot = ring + (size_t)slot_p * FILTER_SLOT;
+                const int i0 = cp * FILTER_CHUNK;
+                uint32_t lastT = filter_half(C, slot, 0, i0, R, tminlo, lane);
+                if (full || lastT <= lmin) lastT = filter_half(C, slot, 64, i0, R, tminlo, lane);
+                finished = !full && lastT > lmin;                  // rows are sorted: nothing later is <= lmin
+            }
+            __syncwarp();
+            --inflight;
+            slot_p = slot_p + 1 == FILTER_STAGES ? 0 : slot_p + 1;
+            if (++cp == req_p) {
+                if (!finished && !full && cp < nchunks) {
+                    // the request ended before the row did: continue with plain loads
+                    for (int i0 = cp * FILTER_CHUNK; i0 < R; i0 += 64) {
+                        const int i = i0 + 2 * lane;
+                        const bool va = i < R, vb = i + 1 < R;
+                        const uint32_t Ta = va ? (uint32_t)(uint64_t)ldg64(row_p + i) - tminlo : 0xffffffffu;
+                        const uint32_t Tb = vb ? (uint32_t)(uint64_t)ldg64(row_p + i + 1) - tminlo : 0xffffffffu;
+                        uint32_t nb = __shfl_down_sync(FULL, Ta, 1);
+                        if (lane == 31) nb = i + 2 < R ? (uint32_t)(uint64_t)ldg64(row_p + i + 2) - tminlo : 0xffffffffu;
+                        filter_pair(C, lane, va, Ta, Tb, vb, Tb, nb);
+                        if (__shfl_sync(FULL, Tb, 31) > lmin) break;
+                    }
+                }
+                cp = 0; ++jp; row_p += rstride; finished = false;
+                req_p = __shfl_sync(FULL, req, min(jp, 31));
+            }
         }
     }
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned c = scount;
+        *rc = min(c, (unsigned)F.regcap);
+        if (c > (unsigned)F.regcap) meta[b].overflow = 1;
+        if (c) atomicAdd(&meta[b].count, c);
+    }
+}
+
+// ------------------------------------------------------------------------------ refinement (RANGE)
+// The per-cell maxima of the filter pass give G exactly at every cell start (the survivors contain every
+// element that ever raises the running maximum).  A survivor whose `next` does not exceed G at the start
+// of its own cell cannot matter either, so it is dropped; the rest go to their time bucket.
+__global__ void __launch_bounds__(1024) k_refine(InstMeta *meta, FilterBufs F) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ uint64_t tmp[34];
+    uint32_t *g = (uint32_t *)smem;                               // exclusive prefix max of cellmax, floored by t0
+    const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+    const InstMeta M = meta[b];
+    if (M.status != ZL_OK || !handled_by_filter(M, 1)) return;
+    const uint32_t m = F.rcnt[(size_t)b * F.nreg + blockIdx.x];
+    if (m == 0) return;
+    const uint32_t cells = (uint32_t)F.cells;
+    const uint32_t *cmx = F.cellmax + (size_t)b * cells;
+    const int per = (int)((cells + nt - 1) / nt);
+    const uint32_t c0 = (uint32_t)tid * per, c1 = min(c0 + per, cells);
+    uint32_t loc = 0;
+    for (uint32_t c = c0; c < c1; ++c) { const uint32_t v = cmx[c]; g[c] = v; loc = max(loc, v); }
+    uint32_t tot;
+    uint32_t run = max(block_scan_excl<uint32_t>(loc, OpMax(), 0u, (uint32_t *)tmp, &tot), (uint32_t)M.t0);
+    for (uint32_t c = c0; c < c1; ++c) { const uint32_t v = g[c]; g[c] = run; run = max(run, v); }
+    __syncthreads();
+    const uint64_t *src = F.list1 + (size_t)b * F.list1cap + (size_t)blockIdx.x * F.regcap;
+    uint32_t *bcnt = F.bcnt + (size_t)b * F.nbk;
+    uint64_t *dst = F.list2 + (size_t)b * F.nbk * F.capb;
+    const int cpb_shift = __ffs(F.cells / F.nbk) - 1;             // cells per bucket is a power of two
+    unsigned kept = 0;
+    bool over = false;
+    for (uint32_t i = tid; i < m; i += nt) {
+        const uint64_t w = src[i];
+        const uint32_t T = (uint32_t)(w >> 32), nx = (uint32_t)w;
+        const uint32_t c = cell_of(T, M.cscale);
+        if (nx > max(T, g[c])) {
+            const uint32_t bk = c >> cpb_shift;
+            const uint32_t pos = atomicAdd(&bcnt[bk], 1u);
+            if (pos < (uint32_t)F.capb) dst[(size_t)bk * F.capb + pos] = w; else over = true;
+            ++kept;
+        }
+    }
+    kept = warp_reduce(kept, OpAdd());
+    if (lane == 0 && kept) atomicAdd(&meta[b].count2, kept);
+    if (over) meta[b].overflow = 1;
 }
 
 // Optional full check that every row is non-decreasing.
@@ -244,7 +445,7 @@ template <typename K, int OBJ>
 __device__ void run_batch(Key<K> *keys, int m, K t0, int n, uint64_t *tmp64, K carryMax, uint64_t &carryS,
                           uint32_t &carryC, uint64_t &bd, uint64_t &bt) {
     if (m == 0) return;
-    int P = 32;
+    int P = 64;
     while (P < m) P <<= 1;
     for (int i = m + threadIdx.x; i < P; i += blockDim.x) keys[i] = Key<K>::inf();
     __syncthreads();
@@ -333,7 +534,7 @@ struct SweepShared {
 
 template <typename K, int OBJ>
 __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int64_t *inst, SweepShared &sh,
-                              uint32_t *curA, uint32_t *curB, Key<K> *keys, SegResult &out) {
+                              uint32_t *curA, uint32_t *curB, Key<K> *keys, int seg_index, SegResult &out) {
     const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
     const int n = P.n, R = P.R, G = P.G, NG = nt / G;
     const int gi = tid / G, g = tid % G;
@@ -347,7 +548,7 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
     const bool cut = OBJ == ZL_OBJ_RANGE && !(P.flags & ZL_FLAG_FULL_SWEEP);
     const uint64_t tend = cut ? M.lmin : M.tend;
     const uint64_t width = (tend + P.nseg - 1) / P.nseg;
-    const uint64_t seg_lo = 1 + (uint64_t)blockIdx.x * width;
+    const uint64_t seg_lo = 1 + (uint64_t)seg_index * width;
     const uint64_t seg_hi = min(seg_lo + width, tend + 1);
     uint64_t bd = ~0ull, bt = ~0ull;          // per-thread best (objective, time)
     uint32_t status = ZL_OK;
@@ -357,7 +558,7 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
     __syncthreads();
     if (seg_lo <= tend) {
         // ---- carry-in: per-row lower bound of the segment start
-        if (blockIdx.x == 0) {
+        if (seg_index == 0) {
             for (int r = tid; r < n; r += nt) curA[r] = 0;
         } else {
             const int64_t a_raw = tmin + (int64_t)(seg_lo - 1);
@@ -519,91 +720,145 @@ template <int OBJ>
 __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ SweepShared sh;
-    const int b = blockIdx.y;
-    const InstMeta M = P.meta[b];
-    SegResult &out = P.seg[(size_t)b * P.nseg + blockIdx.x];
-    if (handled_by_filter(M, P.listcap)) return;             // k_small wrote this instance's result
-    if (M.status != ZL_OK) {
-        if (threadIdx.x == 0) { out.d = ~0ull; out.t = ~0ull; out.valid = 0; out.status = ZL_OK; }
-        return;
-    }
     uint32_t *curA = (uint32_t *)smem;
     uint32_t *curB = curA + P.n;
     unsigned char *kb = smem + (((size_t)2 * P.n * sizeof(uint32_t) + 15) & ~(size_t)15);
-    const int64_t *inst = P.ts + (size_t)b * P.n * P.R;
-    if (M.use32) {
-        sweep_segment<uint32_t, OBJ>(P, M, inst, sh, curA, curB, (Key<uint32_t> *)kb, out);
-    } else {
-        SweepParams Q = P;
-        Q.cap = P.cap / 2;                      // 16-byte nodes: half as many fit
-        sweep_segment<uint64_t, OBJ>(Q, M, inst, sh, curA, curB, (Key<uint64_t> *)kb, out);
+    // a fixed number of CTAs walks the (instance, segment) pairs
+    const int items = P.B * P.nseg;
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        const int b = item / P.nseg, sidx = item % P.nseg;
+        const InstMeta M = P.meta[b];
+        if (handled_by_filter(M, P.filter)) continue;            // the bucket sweep wrote this instance's results
+        SegResult &out = P.seg[(size_t)b * P.nres + sidx];
+        if (M.status != ZL_OK) {
+            if (threadIdx.x == 0) { out.d = ~0ull; out.t = ~0ull; out.valid = 0; out.status = ZL_OK; }
+            continue;
+        }
+        const int64_t *inst = P.ts + (size_t)b * P.n * P.R;
+        if (M.use32) {
+            sweep_segment<uint32_t, OBJ>(P, M, inst, sh, curA, curB, (Key<uint32_t> *)kb, sidx, out);
+        } else {
+            SweepParams Q = P;
+            Q.cap = P.cap / 2;                      // 16-byte nodes: half as many fit
+            sweep_segment<uint64_t, OBJ>(Q, M, inst, sh, curA, curB, (Key<uint64_t> *)kb, sidx, out);
+        }
+        __syncthreads();
     }
 }
 
-// Sort and sweep the filtered list of an instance in one CTA.
-__global__ void __launch_bounds__(1024) k_small(InstMeta *meta, const uint64_t *list_all, uint32_t listcap, int n,
-                                                int nseg, SegResult *seg) {
+// Sort and sweep the refined survivors.  CTA (g, b) takes buckets [g*grp, (g+1)*grp) of instance b in
+// time order, packs whole buckets into shared-memory batches and runs each batch with the running
+// maximum of `next` over everything before it (the prefix maximum of cellmax up to the batch's first cell).
+__global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg) {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
-    __shared__ unsigned int sstatus;
-    const int b = blockIdx.x, tid = threadIdx.x;
+    __shared__ unsigned int sstatus, fill;
+    const int b = blockIdx.y, g = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     const InstMeta M = meta[b];
-    if (M.status != ZL_OK || !handled_by_filter(M, listcap)) return;
+    if (M.status != ZL_OK || !handled_by_filter(M, 1)) return;
     Key<uint32_t> *keys = (Key<uint32_t> *)smem;
-    const uint64_t *list = list_all + (size_t)b * listcap;
-    const int m = (int)M.count;
-    for (int i = tid; i < m; i += blockDim.x) keys[i].w = list[i];
-    if (tid == 0) sstatus = 0;
-    __syncthreads();
+    const uint32_t *bcnt = F.bcnt + (size_t)b * F.nbk;
+    const uint32_t *cmx = F.cellmax + (size_t)b * F.cells;
+    const uint64_t *list = F.list2 + (size_t)b * F.nbk * F.capb;
+    const int grp = bucket_group(F, M.count2);
+    if (g * grp >= F.nbk) return;                                // fewer, wider groups than CTAs for this instance
+    const int first = g * grp, last = min(first + grp, F.nbk);
+    const int cpb = F.cells / F.nbk;
+    if (tid == 0) { sstatus = 0; fill = 0; }
+    // running max of next over everything before the group's first cell
+    uint32_t cm = 0;
+    for (int c = tid; c < first * cpb; c += nt) cm = max(cm, cmx[c]);
+    uint32_t carry0;
+    block_scan_excl<uint32_t>(cm, OpMax(), 0u, (uint32_t *)tmp, &carry0);
     uint64_t bd = ~0ull, bt = ~0ull, cs = 0;
     uint32_t cc = 0;
-    run_batch<uint32_t, ZL_OBJ_RANGE>(keys, m, (uint32_t)M.t0, n, tmp, (uint32_t)0, cs, cc, bd, bt);
-    block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nseg]);
+    uint32_t mine = 0;
+    for (int k = first + tid; k < last; k += nt) mine += min(bcnt[k], (uint32_t)F.capb);
+    uint32_t group_total;
+    block_scan_excl<uint32_t>(mine, OpAdd(), 0u, (uint32_t *)tmp, &group_total);
+    if (group_total <= (uint32_t)F.capb) {
+        // one batch: warps copy whole buckets side by side; offsets come from a running count
+        const int lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+        for (int k = first + warp; k < last; k += nw) {
+            const uint32_t c = min(bcnt[k], (uint32_t)F.capb);
+            if (c == 0) continue;
+            uint32_t off = 0;
+            if (lane == 0) off = atomicAdd(&fill, c);
+            off = __shfl_sync(FULL, off, 0);
+            const uint64_t *src = list + (size_t)k * F.capb;
+            for (uint32_t i = lane; i < c; i += 32) keys[off + i].w = src[i];
+        }
+        __syncthreads();
+        run_batch<uint32_t, ZL_OBJ_RANGE>(keys, (int)group_total, (uint32_t)M.t0, n, tmp, carry0, cs, cc, bd, bt);
+    } else {
+        int m = 0, kstart = first;               // the current batch holds buckets [kstart, k)
+        uint32_t carry_batch = carry0;
+        for (int k = first; k < last; ++k) {
+            const int c = (int)min(bcnt[k], (uint32_t)F.capb);
+            if (c == 0) continue;
+            if (m + c > F.capb) {
+                run_batch<uint32_t, ZL_OBJ_RANGE>(keys, m, (uint32_t)M.t0, n, tmp, carry_batch, cs, cc, bd, bt);
+                // advance the carry over the cells of the buckets just processed
+                uint32_t part = 0, ptot;
+                for (int cidx = kstart * cpb + tid; cidx < k * cpb; cidx += nt) part = max(part, cmx[cidx]);
+                block_scan_excl<uint32_t>(part, OpMax(), 0u, (uint32_t *)tmp, &ptot);
+                carry_batch = max(carry_batch, ptot);
+                kstart = k;
+                m = 0;
+            }
+            const uint64_t *src = list + (size_t)k * F.capb;
+            for (int i = tid; i < c; i += nt) keys[m + i].w = src[i];
+            m += c;
+            __syncthreads();
+        }
+        if (m > 0) run_batch<uint32_t, ZL_OBJ_RANGE>(keys, m, (uint32_t)M.t0, n, tmp, carry_batch, cs, cc, bd, bt);
+    }
+    block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres + g]);
 }
 
 // ------------------------------------------------------------------------------ finalize
-__global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int R, int nseg, int objective,
-                                                  uint32_t listcap, const InstMeta *meta, const SegResult *seg,
+// grid (row blocks, B): every CTA reduces the instance's partial results, then recovers the indices of
+// its block of rows; the CTA of row block 0 also writes wait, barrier and status.
+__global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int R, int nseg, FilterBufs F, int nres,
+                                                  int objective, int filter, const InstMeta *meta, const SegResult *seg,
                                                   int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
-    const int b = blockIdx.x;
+    const int b = blockIdx.y, tid = threadIdx.x;
     const InstMeta M = meta[b];
-    __shared__ int64_t s_barrier;
-    __shared__ int s_status;
-    if (threadIdx.x == 0) {
-        int st = M.status;
-        uint64_t bd = ~0ull, bt = ~0ull;
-        bool have = false;
-        if (st == ZL_OK) {
-            const int nseg_used = handled_by_filter(M, listcap) ? 1 : nseg;
-            for (int s = 0; s < nseg_used; ++s) {
-                const SegResult r = seg[(size_t)b * nseg + s];
-                if (r.status != ZL_OK) st = max(st, r.status);
-                if (!r.valid) continue;
-                if (!have || r.d < bd || (r.d == bd && r.t < bt)) { bd = r.d; bt = r.t; have = true; }
-            }
-            if (st == ZL_OK && !have) st = ZL_ERR_TIMEOUT;     // cannot happen for valid input
-        }
-        if (st == ZL_OK) {
-            const int64_t tm = M.tmin + (int64_t)(bt - 1);
-            s_barrier = objective == ZL_OBJ_RANGE ? tm + (int64_t)bd : tm;
-            wait[b] = (int64_t)bd;
-            barrier[b] = s_barrier;
-        } else {
-            wait[b] = INT64_MIN;
-            barrier[b] = INT64_MIN;
-            s_barrier = INT64_MIN;
-        }
-        s_status = st;
-        if (status) status[b] = st;
-    }
+    __shared__ uint64_t red[34];
+    __shared__ unsigned int sstatus;
+    __shared__ SegResult best;
+    if (tid == 0) sstatus = 0;
     __syncthreads();
-    const int64_t bar = s_barrier;
-    const bool ok = s_status == ZL_OK;
-    const int64_t *inst = ts + (size_t)b * n * R;
-    for (int p = threadIdx.x; p < n; p += blockDim.x) {
+    uint64_t bd = ~0ull, bt = ~0ull;
+    uint32_t st = M.status;
+    if (st == ZL_OK) {
+        const int used = handled_by_filter(M, filter) ? (F.nbk + bucket_group(F, M.count2) - 1) / bucket_group(F, M.count2) : nseg;
+        for (int s = tid; s < used; s += blockDim.x) {
+            const SegResult r = seg[(size_t)b * nres + s];
+            if (r.status != ZL_OK) st = max(st, (uint32_t)r.status);
+            if (r.valid && (r.d < bd || (r.d == bd && r.t < bt))) { bd = r.d; bt = r.t; }
+        }
+    }
+    block_best_to_result(bd, bt, st, red, &sstatus, best);
+    __syncthreads();
+    int fst = (int)best.status;
+    if (fst == ZL_OK && !best.valid) fst = ZL_ERR_TIMEOUT;         // cannot happen for valid input
+    int64_t bar = INT64_MIN, wt = INT64_MIN;
+    if (fst == ZL_OK) {
+        const int64_t tm = M.tmin + (int64_t)(best.t - 1);
+        bar = objective == ZL_OBJ_RANGE ? tm + (int64_t)best.d : tm;
+        wt = (int64_t)best.d;
+    }
+    if (blockIdx.x == 0 && tid == 0) {
+        wait[b] = wt;
+        barrier[b] = bar;
+        if (status) status[b] = fst;
+    }
+    const int p = blockIdx.x * blockDim.x + tid;
+    if (p < n) {
         int res = -1;
-        if (ok) {
-            const int64_t *row = inst + (size_t)p * R;
+        if (fst == ZL_OK) {
+            const int64_t *row = ts + ((size_t)b * n + p) * R;
             int lo = 0, hi = R;                   // number of elements <= barrier
             while (lo < hi) {
                 const int mid = (lo + hi) >> 1;
@@ -630,7 +885,7 @@ __global__ void __launch_bounds__(256) k_trace(const int64_t *ts, int n, int R,
     TKey *keys = (TKey *)smem;
     const int N = n * R, b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     const int64_t *inst = ts + (size_t)b * N;
-    int P = 32;
+    int P = 64;
     while (P < N) P <<= 1;
     // step 1: merge = all (time, worker, iteration) in ascending order
     int64_t t0loc = INT64_MIN;
@@ -700,9 +955,8 @@ struct zl_handle {
     int num_sms;
     zl::InstMeta *d_meta;
     zl::SegResult *d_seg;
-    uint32_t *d_table;       // RANGE: filter tables, [max_batch][max_cells]
-    uint64_t *d_list;        // RANGE: filtered (T, next) lists, [max_batch][listcap]
-    int max_cells, listcap;
+    zl::FilterBufs fb;       // RANGE: buffers of the filter route (device), sized for max_batch
+    int nres;                // SegResult slots per instance
     size_t ws_bytes;
     // host-buffer path
     int64_t *s_ts; int32_t *s_idx; int64_t *s_barrier; int64_t *s_wait; int32_t *s_status;
@@ -728,16 +982,18 @@ constexpr int PROF_EVENTS = 5;
 // Everything one call enqueues, for both the handle-based and the fixed-scratch entry points.
 struct Pipeline {
     const int64_t *ts; int B, n, R, objective, flags, num_sms;
-    zl::InstMeta *meta; zl::SegResult *seg;
-    uint32_t *table; uint64_t *list; int max_cells, listcap;      // table == nullptr: no filter path
+    zl::InstMeta *meta; zl::SegResult *seg; int nres;
+    zl::FilterBufs fb;                                            // fb.table == nullptr: no filter route
     int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;
 };
 
 void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_t *ev) {
-    const bool filter = q.table != nullptr && q.objective == ZL_OBJ_RANGE;
-    const uint32_t listcap = filter ? (uint32_t)q.listcap : 0u;
+    const bool filter = q.fb.table != nullptr && q.objective == ZL_OBJ_RANGE;
+    zl::FilterBufs fb = q.fb;
+    if (!filter) memset(&fb, 0, sizeof(fb));
     if (ev) cudaEventRecord(ev[0], st);
-    zl::k_prologue<<<q.B, 1024, 0, st>>>(q.ts, q.n, q.R, q.objective, q.flags, q.meta, filter ? q.table : nullptr, q.max_cells);
+    const int pthreads = std::max(128, std::min(1024, pow2_ceil(q.n)));
+    zl::k_prologue<<<q.B, pthreads, 0, st>>>(q.ts, q.n, q.R, q.objective, q.flags, q.meta, fb);
     if (q.flags & ZL_FLAG_CHECK_SORTED) {
         const size_t total = (size_t)q.B * q.n * q.R;
         const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)q.num_sms * 16);
@@ -749,31 +1005,40 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         const int nw = threads / 32;
         long long rpc = ((long long)q.n * q.B / (4LL * q.num_sms) + nw - 1) / nw * nw;
         rpc = std::max<long long>(nw, std::min<long long>(rpc, (q.n + nw - 1) / nw * nw));
-        const dim3 grid((unsigned)((q.n + rpc - 1) / rpc), q.B);
-        zl::k_filter<<<grid, threads, (size_t)q.max_cells * 4, st>>>(q.ts, q.n, q.R, q.flags, (int)rpc, q.meta, q.table,
-                                                                   q.max_cells, q.list, listcap);
-    }
-    if (ev) cudaEventRecord(ev[2], st);
-    if (filter) {
-        const int threads = std::max(128, std::min(1024, q.listcap / 4));
-        zl::k_small<<<q.B, threads, (size_t)q.listcap * 8, st>>>(q.meta, q.list, listcap, q.n, p.nseg, q.seg);
+        fb.nreg = (int)((q.n + rpc - 1) / rpc);
+        fb.regcap = fb.list1cap / fb.nreg;
+        const size_t fsmem = (size_t)fb.cells * 4 + (size_t)nw * zl::FILTER_STAGES * zl::FILTER_SLOT * 8;
+        zl::k_filter<<<dim3(fb.nreg, q.B), threads, fsmem, st>>>(q.ts, q.n, q.R, q.flags, (int)rpc, q.meta, fb);
+        if (ev) cudaEventRecord(ev[2], st);
+        const int rthreads = std::max(128, std::min(1024, fb.cells / 4));
+        zl::k_refine<<<dim3(fb.nreg, q.B), rthreads, (size_t)fb.cells * 4, st>>>(q.meta, fb);
+        const int ngroups = (fb.nbk + fb.grp - 1) / fb.grp;
+        const int bthreads = std::max(64, std::min(256, fb.capb / 4));
+        zl::k_buckets<<<dim3(ngroups, q.B), bthreads, (size_t)fb.capb * 8, st>>>(q.meta, fb, q.n, q.nres, q.seg);
+    } else if (ev) {
+        cudaEventRecord(ev[2], st);
     }
     zl::SweepParams sp;
     sp.ts = q.ts; sp.meta = q.meta; sp.seg = q.seg;
-    sp.n = q.n; sp.R = q.R; sp.nseg = p.nseg; sp.G = p.G; sp.cap = p.cap; sp.flags = q.flags; sp.target = p.target;
-    sp.listcap = listcap;
-    const dim3 grid(p.nseg, q.B);
-    if (q.objective == ZL_OBJ_RANGE) zl::k_sweep<ZL_OBJ_RANGE><<<grid, p.threads, p.smem, st>>>(sp);
-    else zl::k_sweep<ZL_OBJ_SUM><<<grid, p.threads, p.smem, st>>>(sp);
+    sp.n = q.n; sp.R = q.R; sp.B = q.B; sp.nseg = p.nseg; sp.nres = q.nres; sp.G = p.G; sp.cap = p.cap;
+    sp.flags = q.flags; sp.target = p.target; sp.filter = filter ? 1 : 0;
+    // with the filter route on, the segment sweep is only the fallback: a small persistent grid
+    const int items = p.nseg * q.B;
+    const int sweep_ctas = filter ? std::min(items, 2 * q.num_sms) : items;
+    if (q.objective == ZL_OBJ_RANGE) zl::k_sweep<ZL_OBJ_RANGE><<<sweep_ctas, p.threads, p.smem, st>>>(sp);
+    else zl::k_sweep<ZL_OBJ_SUM><<<sweep_ctas, p.threads, p.smem, st>>>(sp);
     if (ev) cudaEventRecord(ev[3], st);
-    zl::k_finalize<<<q.B, 256, 0, st>>>(q.ts, q.n, q.R, p.nseg, q.objective, listcap, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
+    zl::k_finalize<<<dim3((q.n + 255) / 256, q.B), 256, 0, st>>>(q.ts, q.n, q.R, p.nseg, fb, q.nres, q.objective,
+                                                                  filter ? 1 : 0, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
     if (ev) cudaEventRecord(ev[4], st);
 }
 
 cudaError_t raise_shared_memory_limits() {
     cudaError_t e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_small, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_buckets, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_refine, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     return e;
 }
 
@@ -787,7 +1052,7 @@ LaunchPlan make_plan(const zl_handle *h, int B) {
     // batch capacity in 8-byte nodes; wide (16-byte) instances get half, which must still hold one
     // node per worker
     int cap = std::max(8192, pow2_ceil(2 * n));
-    const int small = std::max(pow2_ceil((int)std::min<long long>(N, 1 << 20)), std::max(pow2_ceil(2 * n), 64));
+    const int small = std::max(pow2_ceil((int)std::min<long long>(N, 1 << 20)), std::max(pow2_ceil(2 * n), 128));
     p.cap = std::min(cap, small);
     // time segments per instance: enough CTAs to fill the GPU a few times over, each long enough to
     // amortise its binary searches
@@ -853,27 +1118,40 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     cudaError_t e = cudaSetDevice(cfg->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, cfg->device);
     const size_t meta_b = (size_t)cfg->max_batch * sizeof(zl::InstMeta);
-    const size_t seg_b = (size_t)cfg->max_batch * zl::MAX_SEGMENTS * sizeof(zl::SegResult);
-    if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_meta, meta_b);
-    if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_seg, seg_b);
-    size_t table_b = 0, list_b = 0;
+    size_t filter_b = 0;
+    h->nres = zl::MAX_SEGMENTS;
     if (cfg->objective == ZL_OBJ_RANGE) {
         const long long N = (long long)cfg->n_workers * cfg->lookahead_R;
-        h->max_cells = std::max(64, std::min(zl::FILTER_MAX_CELLS, pow2_ceil((int)std::min<long long>(4LL * cfg->lookahead_R, 1 << 20))));
-        h->listcap = std::max(64, std::min(16384, pow2_ceil((int)std::min<long long>(N, 1 << 20))));
-        table_b = (size_t)cfg->max_batch * h->max_cells * sizeof(uint32_t);
-        list_b = (size_t)cfg->max_batch * h->listcap * sizeof(uint64_t);
-        if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_table, table_b);
-        if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_list, list_b);
+        const size_t mb = (size_t)cfg->max_batch;
+        zl::FilterBufs &f = h->fb;
+        f.cells = std::max(64, std::min(zl::FILTER_MAX_CELLS, pow2_ceil((int)std::min<long long>(4LL * cfg->lookahead_R, 1 << 20))));
+        f.capb = (int)std::max<long long>(64, std::min<long long>(4096, pow2_ceil((int)std::min<long long>(N, 1 << 20))));
+        f.nbk = (int)std::max<long long>(1, std::min<long long>(std::min(1024, f.cells), pow2_ceil((int)std::min<long long>(N / 8 / f.capb, 1 << 20))));
+        f.grp = std::max(1, std::min(f.nbk, pow2_floor((int)std::max<long long>(1, (long long)f.nbk * cfg->max_batch / (8LL * std::max(1, h->num_sms))))));
+        f.list1cap = (int)std::max<long long>(N / 2, std::min<long long>(N, 4096));
+        h->nres = std::max(zl::MAX_SEGMENTS, (f.nbk + f.grp - 1) / f.grp);
+        const size_t sizes[7] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.cells * 4, mb * cfg->n_workers * 4,
+                                 mb * (size_t)f.list1cap * 8, mb * f.nbk * 4, mb * f.nbk * f.capb * 8};
+        void **ptrs[7] = {(void **)&f.table, (void **)&f.rowhint, (void **)&f.cellmax, (void **)&f.rcnt,
+                          (void **)&f.list1, (void **)&f.bcnt, (void **)&f.list2};
+        for (int i = 0; i < 7; ++i) {
+            if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
+            filter_b += sizes[i];
+        }
     }
+    const size_t seg_b = (size_t)cfg->max_batch * h->nres * sizeof(zl::SegResult);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_meta, meta_b);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_seg, seg_b);
     if (e == cudaSuccess) e = raise_shared_memory_limits();   // more than the default 48 KB of dynamic shared memory
     if (e != cudaSuccess) {
         zl_status st = cuda_fail(nullptr, e);
-        cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_table); cudaFree(h->d_list);
+        cudaFree(h->d_meta); cudaFree(h->d_seg);
+        cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
+        cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2);
         delete h;
         return st;
     }
-    h->ws_bytes = meta_b + seg_b + table_b + list_b;
+    h->ws_bytes = meta_b + seg_b + filter_b;
     *out = h;
     return ZL_OK;
 }
@@ -929,7 +1207,9 @@ zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_stage) {
 zl_status zl_destroy(zl_handle *h) {
     if (!h) return ZL_OK;
     cudaSetDevice(h->cfg.device);
-    cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_table); cudaFree(h->d_list);
+    cudaFree(h->d_meta); cudaFree(h->d_seg);
+    cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
+    cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2);
     cudaFree(h->s_ts); cudaFree(h->s_idx); cudaFree(h->s_barrier); cudaFree(h->s_wait); cudaFree(h->s_status);
     if (h->s_stream) cudaStreamDestroy(h->s_stream);
     zl_profile_end(h);
@@ -964,7 +1244,7 @@ size_t zl_workspace_bytes(const zl_handle *h) { return h ? h->ws_bytes + h->stag
 int32_t zl_launches_per_call(const zl_handle *h) {
     if (!h) return 0;
     const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter;
-    return 3 + (filter ? 2 : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
+    return 3 + (filter ? 3 : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
 }
 int32_t zl_segments_per_instance(const zl_handle *h, int32_t B) { return h && B >= 1 ? make_plan(h, B).nseg : 0; }
 int32_t zl_last_cuda_error(const zl_handle *h) { return h ? h->last_cuda_error : 0; }
@@ -984,13 +1264,27 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     cudaEvent_t *ev = (h->prof_ev && h->prof_calls < h->prof_cap) ? h->prof_ev + PROF_EVENTS * (size_t)h->prof_calls : nullptr;
     Pipeline q;
     q.ts = d_ts; q.B = B; q.n = n; q.R = R; q.objective = obj; q.flags = h->cfg.flags; q.num_sms = h->num_sms;
-    q.meta = h->d_meta; q.seg = h->d_seg;
-    q.table = h->opt_no_filter ? nullptr : h->d_table; q.list = h->d_list; q.max_cells = h->max_cells; q.listcap = h->listcap;
+    q.meta = h->d_meta; q.seg = h->d_seg; q.nres = h->nres;
+    q.fb = h->fb;
+    if (h->opt_no_filter) q.fb.table = nullptr;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, st, ev);
     if (ev) ++h->prof_calls;
     ZL_CUDA(h, cudaGetLastError());
     h->launches += zl_launches_per_call(h);
+    return ZL_OK;
+}
+
+zl_status zl_filter_counts(zl_handle *h, int32_t B, uint32_t *h_filtered, uint32_t *h_refined, uint32_t *h_overflow) {
+    if (!h || B < 1 || B > h->cfg.max_batch) return ZL_ERR_INVALID_ARG;
+    ZL_CUDA(h, cudaSetDevice(h->cfg.device));
+    ZL_CUDA(h, cudaDeviceSynchronize());
+    uint32_t *dst[3] = {h_filtered, h_refined, h_overflow};
+    const size_t off[3] = {offsetof(zl::InstMeta, count), offsetof(zl::InstMeta, count2), offsetof(zl::InstMeta, overflow)};
+    for (int i = 0; i < 3; ++i)
+        if (dst[i])
+            ZL_CUDA(h, cudaMemcpy2D(dst[i], sizeof(uint32_t), (const char *)h->d_meta + off[i], sizeof(zl::InstMeta),
+                                    sizeof(uint32_t), (size_t)B, cudaMemcpyDeviceToHost));
     return ZL_OK;
 }
 
@@ -1026,7 +1320,7 @@ zl_status zl_trace_batched(const int64_t *d_ts, int32_t B, int32_t n, int32_t R,
                            int64_t *PM, int64_t *d_range, int64_t *w_sum, void *cuda_stream) {
     if (!d_ts || B < 1 || n < 1 || R < 1) return ZL_ERR_INVALID_ARG;
     if ((long long)n * R > zl::TRACE_MAX) return ZL_ERR_UNSUPPORTED;
-    const int P = std::max(32, pow2_ceil(n * R));
+    const int P = std::max(64, pow2_ceil(n * R));
     const size_t smem = (size_t)P * sizeof(zl::TKey);
     cudaError_t e = cudaFuncSetAttribute(zl::k_trace, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(zl::TRACE_MAX * sizeof(zl::TKey)));
     if (e != cudaSuccess) return ZL_ERR_CUDA;
@@ -1110,8 +1404,8 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     // never read.  (The filter path of the handle-based entry point needs two more buffers and is not used here.)
     Pipeline q;
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
-    q.meta = meta; q.seg = seg;
-    q.table = nullptr; q.list = nullptr; q.max_cells = 0; q.listcap = 0;
+    q.meta = meta; q.seg = seg; q.nres = p.nseg;
+    memset(&q.fb, 0, sizeof(q.fb));
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr);
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;

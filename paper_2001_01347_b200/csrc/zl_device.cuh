@@ -38,21 +38,36 @@ template <> __device__ __forceinline__ uint32_t kinf<uint32_t>() { return 0xffff
 template <> __device__ __forceinline__ uint64_t kinf<uint64_t>() { return ~0ull; }
 
 // ---------------------------------------------------------------------------------- sort
-// Ascending bitonic sort of keys[0..P) in shared memory, P a power of two, by the whole block.
+// Ascending bitonic sort of keys[0..P) in shared memory, P a power of two >= 64, by the whole block
+// (blockDim a multiple of 32).  Compare-exchange steps with distance j <= 32 stay inside the 64-key
+// block that a warp's 32 consecutive pair indices cover, so runs of such steps are separated by
+// __syncwarp() only; steps with a larger distance need the block barrier.
+template <typename KeyT>
+__device__ __forceinline__ void bitonic_step(KeyT *keys, int i, int j, int k) {
+    const int lo = ((i & ~(j - 1)) << 1) | (i & (j - 1));
+    const int hi = lo | j;
+    const bool up = (lo & k) == 0;
+    KeyT x = keys[lo], y = keys[hi];
+    if ((x > y) == up) { keys[lo] = y; keys[hi] = x; }
+}
+
 template <typename KeyT>
 __device__ void bitonic_sort(KeyT *keys, int P) {
-    const int tid = threadIdx.x, nt = blockDim.x;
+    const int tid = threadIdx.x, nt = blockDim.x, half = P >> 1;
     for (int k = 2; k <= P; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = tid; i < (P >> 1); i += nt) {
-                const int lo = ((i & ~(j - 1)) << 1) | (i & (j - 1));
-                const int hi = lo | j;
-                const bool up = (lo & k) == 0;
-                KeyT x = keys[lo], y = keys[hi];
-                if ((x > y) == up) { keys[lo] = y; keys[hi] = x; }
-            }
+        int j = k >> 1;
+        for (; j > 32; j >>= 1) {
+            for (int i = tid; i < half; i += nt) bitonic_step(keys, i, j, k);
             __syncthreads();
         }
+        // j <= 32: each warp finishes its own 64-key blocks
+        for (int i0 = tid; i0 < half; i0 += nt) {
+            for (int jj = j; jj > 0; jj >>= 1) {
+                bitonic_step(keys, i0, jj, k);
+                __syncwarp();
+            }
+        }
+        __syncthreads();
     }
 }
 
