@@ -39,9 +39,11 @@ struct InstMeta {
     int32_t use32;       // relative times fit 32 bits
     uint32_t cscale;     // filter route: time cell of relative time T = ((T - 1) * cscale) >> 32 (monotone in T);
                          // 0: the instance does not take the filter route
+    uint32_t fscale;     // same map onto the fine cells of the refinement
     uint32_t count;      // survivors of the filter pass
     uint32_t count2;     // survivors of the refinement
     uint32_t overflow;   // a survivor list overflowed: the instance takes the segment sweep instead
+    uint32_t pad;
 };
 
 struct SegResult {
@@ -51,17 +53,19 @@ struct SegResult {
     int32_t status;
 };
 
-// Buffers of the RANGE filter route (all nullptr / 0 when the route is off).  Time is cut into
-// `cells` cells per instance; `nbk` buckets are runs of cells / nbk consecutive cells.
+// Buffers of the RANGE filter route (all nullptr / 0 when the route is off).  The time up to lmin is
+// cut into `cells` coarse cells (filter table, shared memory) and `fcells` fine cells (refinement);
+// `nbk` buckets are runs of fcells / nbk consecutive fine cells.
 struct FilterBufs {
     uint32_t *table;     // [B][cells]        lower bound of G at the start of each cell (from a few slow rows)
     uint32_t *rowhint;   // [B][n]            estimated number of elements of a row that are <= lmin
-    uint32_t *cellmax;   // [B][cells]        max `next` over the filter pass's survivors of each cell
+    uint32_t *cellmax;   // [B][fcells]       max `next` over the filter pass's survivors of each fine cell; after
+                         //                   k_cellscan: G at the start of each fine cell
     uint32_t *rcnt;      // [B][nreg]         survivors per region (one region per CTA of the filter pass)
     uint64_t *list1;     // [B][list1cap]     survivors of the filter pass as (T << 32 | next), by region
     uint32_t *bcnt;      // [B][nbk]          survivors of the refinement per bucket
     uint64_t *list2;     // [B][nbk][capb]    survivors of the refinement
-    int32_t cells, nbk, capb, grp;           // grp: fewest buckets per CTA of the bucket sweep
+    int32_t cells, fcells, nbk, capb, grp;   // grp: fewest buckets per CTA of the bucket sweep
     int32_t nreg, regcap, list1cap;          // set per call: regions per instance and their capacity
 };
 
@@ -87,6 +91,11 @@ __device__ __forceinline__ bool handled_by_filter(const InstMeta &M, int filter)
 }
 
 __device__ __forceinline__ uint32_t cell_of(uint32_t T, uint32_t cscale) { return __umulhi(T - 1, cscale); }
+
+// Instances with at most this many survivors of the filter pass are finished by one CTA (k_tail);
+// larger ones go through cell scan, refinement and the bucket sweep.
+constexpr uint32_t TAIL_CAP = 8192;
+__device__ __forceinline__ bool tail_instance(const InstMeta &M) { return M.count <= TAIL_CAP; }
 
 // ------------------------------------------------------------------------------ prologue
 // Column scans per instance, and (RANGE, 32-bit instances) the filter table.
@@ -130,7 +139,7 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
         InstMeta m;
         m.tmin = tmin;
         m.status = ZL_OK;
-        m.cscale = 0; m.count = 0; m.count2 = 0; m.overflow = 0;
+        m.cscale = 0; m.fscale = 0; m.count = 0; m.count2 = 0; m.overflow = 0; m.pad = 0;
         if (tmin < 0 || tmax >= VALUE_LIMIT || tmax < tmin || lmin < tmin) {
             m.status = ZL_ERR_INVALID_ARG;     // outside [0, 2^62), or first/last columns out of order
             m.t0 = m.lmin = m.tend = 1; m.use32 = 1;
@@ -140,9 +149,11 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
             m.tend = (uint64_t)(tmax - tmin) + 1;
             m.use32 = m.tend < 0xfffffffeull;
             if (objective == ZL_OBJ_SUM && m.tend > (uint64_t)INT64_MAX / (uint64_t)n) m.status = ZL_ERR_UNSUPPORTED;
-            if (objective == ZL_OBJ_RANGE && F.table && m.use32 && m.status == ZL_OK)
+            if (objective == ZL_OBJ_RANGE && F.table && m.use32 && m.status == ZL_OK) {
                 // (T - 1) < lmin for every T <= lmin, so ((T - 1) * cscale) >> 32 < cells
                 m.cscale = (uint32_t)max((uint64_t)1, min((uint64_t)0xffffffffu, ((uint64_t)F.cells << 32) / m.lmin));
+                m.fscale = (uint32_t)max((uint64_t)1, min((uint64_t)0xffffffffu, ((uint64_t)F.fcells << 32) / m.lmin));
+            }
         }
         sm = m;
     }
@@ -151,8 +162,9 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
     if (M.cscale != 0) {
         const uint32_t cells = (uint32_t)F.cells, cscale = M.cscale, lmin = (uint32_t)M.lmin;
         const int64_t tmin = M.tmin;
-        uint32_t *cmx = F.cellmax + (size_t)b * cells;
-        for (uint32_t c = tid; c < cells; c += nt) { tab[c] = (uint32_t)M.t0; cmx[c] = 0; }
+        uint32_t *cmx = F.cellmax + (size_t)b * F.fcells;
+        for (uint32_t c = tid; c < cells; c += nt) tab[c] = (uint32_t)M.t0;
+        for (uint32_t c = tid; c < (uint32_t)F.fcells; c += nt) cmx[c] = 0;
         for (int k = tid; k < F.nbk; k += nt) F.bcnt[(size_t)b * F.nbk + k] = 0;
         // per row: how many of its elements are expected to be <= lmin (rows are close to arithmetic);
         // the filter pass uses it only to decide how much of the row to request up front
@@ -183,20 +195,27 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
             const int64_t *rp = inst + (size_t)row * R;
             // element i is the first element of the row at or after every cell start in (e_{i-1}, e_i]:
             // the cells after the one holding e_{i-1}, up to the one holding e_i
-            for (int i0 = 1; i0 < R; i0 += 32) {
-                const int i = i0 + lane;
-                uint32_t prev = 0xffffffffu, curv = 0;
-                if (i < R) {
-                    prev = (uint32_t)(ldg64(rp + i - 1) - tmin + 1);
-                    curv = (uint32_t)(ldg64(rp + i) - tmin + 1);
+            // (four 32-element steps are loaded before any is used: the loop is latency bound otherwise)
+            for (int i0 = 1; i0 < R; i0 += 128) {
+                uint32_t pv[4], cv[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int i = i0 + 32 * k + lane;
+                    pv[k] = 0xffffffffu; cv[k] = 0;
+                    if (i < R) {
+                        pv[k] = (uint32_t)(ldg64(rp + i - 1) - tmin + 1);
+                        cv[k] = (uint32_t)(ldg64(rp + i) - tmin + 1);
+                    }
                 }
-                if (i < R && prev <= lmin) {
-                    const uint32_t c_from = cell_of(prev, cscale) + 1;
-                    const uint32_t c_to = curv <= lmin ? cell_of(curv, cscale) : cells - 1;
-                    for (uint32_t c = c_from; c <= c_to && c < cells; ++c) atomicMax(&tab[c], curv);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (pv[k] <= lmin) {              // also false past the end of the row
+                        const uint32_t c_from = cell_of(pv[k], cscale) + 1;
+                        const uint32_t c_to = cv[k] <= lmin ? cell_of(cv[k], cscale) : cells - 1;
+                        for (uint32_t c = c_from; c <= c_to && c < cells; ++c) atomicMax(&tab[c], cv[k]);
+                    }
                 }
-                const uint32_t first_prev = __shfl_sync(FULL, prev, 0);
-                if (first_prev > lmin) break;                     // the rest of the row lies after lmin
+                if (__shfl_sync(FULL, pv[3], 0) > lmin) break;    // the rest of the row lies after lmin
             }
         }
         __syncthreads();
@@ -240,7 +259,7 @@ __device__ __forceinline__ void cp_async_wait_pending(int pending) {
 
 struct FilterCtx {
     const uint32_t *tab; uint64_t *list; uint32_t *cellmax; unsigned int *scount;
-    uint32_t cscale, lmin, regcap;
+    uint32_t cscale, fscale, lmin, regcap;
 };
 
 // Table test of the (up to) two elements of a lane, warp-aggregated append of the survivors.
@@ -260,12 +279,12 @@ __device__ __forceinline__ void filter_pair(const FilterCtx &c, int lane, bool v
     if (ka) {
         const unsigned pos = base + __popc(ma & below);
         if (pos < c.regcap) c.list[pos] = ((uint64_t)Ta << 32) | na;
-        atomicMax(&c.cellmax[ca], na);
+        atomicMax(&c.cellmax[cell_of(Ta, c.fscale)], na);
     }
     if (kb) {
         const unsigned pos = base + na_cnt + __popc(mb & below);
         if (pos < c.regcap) c.list[pos] = ((uint64_t)Tb << 32) | nb;
-        atomicMax(&c.cellmax[cb], nb);
+        atomicMax(&c.cellmax[cell_of(Tb, c.fscale)], nb);
     }
 }
 
@@ -303,8 +322,8 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
     const bool full = (flags & ZL_FLAG_FULL_SWEEP) != 0;
     FilterCtx C;
     C.tab = tab; C.list = F.list1 + (size_t)b * F.list1cap + (size_t)blockIdx.x * F.regcap;
-    C.cellmax = F.cellmax + (size_t)b * cells; C.scount = &scount;
-    C.cscale = M.cscale; C.lmin = lmin; C.regcap = (uint32_t)F.regcap;
+    C.cellmax = F.cellmax + (size_t)b * F.fcells; C.scount = &scount;
+    C.cscale = M.cscale; C.fscale = M.fscale; C.lmin = lmin; C.regcap = (uint32_t)F.regcap;
     const int r0 = blockIdx.x * rows_per_cta, r1 = min(r0 + rows_per_cta, n);
     const bool vec2 = (R % 2 == 0) && (((uintptr_t)ts & 15) == 0);
     const int nchunks = (R + FILTER_CHUNK - 1) / FILTER_CHUNK;
@@ -384,39 +403,55 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
 }
 
 // ------------------------------------------------------------------------------ refinement (RANGE)
-// The per-cell maxima of the filter pass give G exactly at every cell start (the survivors contain every
-// element that ever raises the running maximum).  A survivor whose `next` does not exceed G at the start
-// of its own cell cannot matter either, so it is dropped; the rest go to their time bucket.
-__global__ void __launch_bounds__(1024) k_refine(InstMeta *meta, FilterBufs F) {
-    extern __shared__ __align__(16) unsigned char smem[];
+// The per-cell maxima of the filter pass give G exactly at every fine cell start (the survivors contain
+// every element that ever raises the running maximum): k_cellscan turns cellmax, in place, into its
+// exclusive prefix maximum floored by t0.  A survivor whose `next` does not exceed G at the start of its
+// own cell cannot matter either, so k_refine drops it; the rest go to their time bucket.
+__global__ void __launch_bounds__(1024) k_cellscan(const InstMeta *meta, FilterBufs F) {
     __shared__ uint64_t tmp[34];
-    uint32_t *g = (uint32_t *)smem;                               // exclusive prefix max of cellmax, floored by t0
+    __shared__ uint32_t tile[4096];
+    const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+    const InstMeta M = meta[b];
+    if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) return;
+    uint32_t *cmx = F.cellmax + (size_t)b * F.fcells;
+    uint32_t carry = (uint32_t)M.t0;
+    // tiles of 4096 cells: coalesced in, each thread scans a run of consecutive cells, coalesced out
+    for (int base = 0; base < F.fcells; base += 4096) {
+        const int len = min(4096, F.fcells - base);
+        for (int i = tid; i < len; i += nt) tile[i] = cmx[base + i];
+        __syncthreads();
+        const int per = (len + nt - 1) / nt;
+        const int c0 = min(tid * per, len), c1 = min(c0 + per, len);
+        uint32_t loc = 0;
+        for (int c = c0; c < c1; ++c) loc = max(loc, tile[c]);
+        uint32_t tot;
+        uint32_t run = max(block_scan_excl<uint32_t>(loc, OpMax(), 0u, (uint32_t *)tmp, &tot), carry);
+        for (int c = c0; c < c1; ++c) { const uint32_t v = tile[c]; tile[c] = run; run = max(run, v); }
+        carry = max(carry, tot);
+        __syncthreads();
+        for (int i = tid; i < len; i += nt) cmx[base + i] = tile[i];
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(1024) k_refine(InstMeta *meta, FilterBufs F) {
     const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
     const InstMeta M = meta[b];
-    if (M.status != ZL_OK || !handled_by_filter(M, 1)) return;
+    if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) return;
     const uint32_t m = F.rcnt[(size_t)b * F.nreg + blockIdx.x];
     if (m == 0) return;
-    const uint32_t cells = (uint32_t)F.cells;
-    const uint32_t *cmx = F.cellmax + (size_t)b * cells;
-    const int per = (int)((cells + nt - 1) / nt);
-    const uint32_t c0 = (uint32_t)tid * per, c1 = min(c0 + per, cells);
-    uint32_t loc = 0;
-    for (uint32_t c = c0; c < c1; ++c) { const uint32_t v = cmx[c]; g[c] = v; loc = max(loc, v); }
-    uint32_t tot;
-    uint32_t run = max(block_scan_excl<uint32_t>(loc, OpMax(), 0u, (uint32_t *)tmp, &tot), (uint32_t)M.t0);
-    for (uint32_t c = c0; c < c1; ++c) { const uint32_t v = g[c]; g[c] = run; run = max(run, v); }
-    __syncthreads();
+    const uint32_t *g = F.cellmax + (size_t)b * F.fcells;         // G at fine cell starts
     const uint64_t *src = F.list1 + (size_t)b * F.list1cap + (size_t)blockIdx.x * F.regcap;
     uint32_t *bcnt = F.bcnt + (size_t)b * F.nbk;
     uint64_t *dst = F.list2 + (size_t)b * F.nbk * F.capb;
-    const int cpb_shift = __ffs(F.cells / F.nbk) - 1;             // cells per bucket is a power of two
+    const int cpb_shift = __ffs(F.fcells / F.nbk) - 1;            // fine cells per bucket is a power of two
     unsigned kept = 0;
     bool over = false;
     for (uint32_t i = tid; i < m; i += nt) {
         const uint64_t w = src[i];
         const uint32_t T = (uint32_t)(w >> 32), nx = (uint32_t)w;
-        const uint32_t c = cell_of(T, M.cscale);
-        if (nx > max(T, g[c])) {
+        const uint32_t c = cell_of(T, M.fscale);
+        if (nx > max(T, __ldg(g + c))) {
             const uint32_t bk = c >> cpb_shift;
             const uint32_t pos = atomicAdd(&bcnt[bk], 1u);
             if (pos < (uint32_t)F.capb) dst[(size_t)bk * F.capb + pos] = w; else over = true;
@@ -755,21 +790,19 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
     __shared__ unsigned int sstatus, fill;
     const int b = blockIdx.y, g = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     const InstMeta M = meta[b];
-    if (M.status != ZL_OK || !handled_by_filter(M, 1)) return;
+    if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) return;
     Key<uint32_t> *keys = (Key<uint32_t> *)smem;
     const uint32_t *bcnt = F.bcnt + (size_t)b * F.nbk;
-    const uint32_t *cmx = F.cellmax + (size_t)b * F.cells;
+    const uint32_t *g0 = F.cellmax + (size_t)b * F.fcells;        // G at fine cell starts (after k_cellscan)
     const uint64_t *list = F.list2 + (size_t)b * F.nbk * F.capb;
     const int grp = bucket_group(F, M.count2);
     if (g * grp >= F.nbk) return;                                // fewer, wider groups than CTAs for this instance
     const int first = g * grp, last = min(first + grp, F.nbk);
-    const int cpb = F.cells / F.nbk;
+    const int cpb = F.fcells / F.nbk;
     if (tid == 0) { sstatus = 0; fill = 0; }
+    __syncthreads();
     // running max of next over everything before the group's first cell
-    uint32_t cm = 0;
-    for (int c = tid; c < first * cpb; c += nt) cm = max(cm, cmx[c]);
-    uint32_t carry0;
-    block_scan_excl<uint32_t>(cm, OpMax(), 0u, (uint32_t *)tmp, &carry0);
+    const uint32_t carry0 = g0[(size_t)first * cpb];
     uint64_t bd = ~0ull, bt = ~0ull, cs = 0;
     uint32_t cc = 0;
     uint32_t mine = 0;
@@ -791,19 +824,14 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
         __syncthreads();
         run_batch<uint32_t, ZL_OBJ_RANGE>(keys, (int)group_total, (uint32_t)M.t0, n, tmp, carry0, cs, cc, bd, bt);
     } else {
-        int m = 0, kstart = first;               // the current batch holds buckets [kstart, k)
+        int m = 0;
         uint32_t carry_batch = carry0;
         for (int k = first; k < last; ++k) {
             const int c = (int)min(bcnt[k], (uint32_t)F.capb);
             if (c == 0) continue;
             if (m + c > F.capb) {
                 run_batch<uint32_t, ZL_OBJ_RANGE>(keys, m, (uint32_t)M.t0, n, tmp, carry_batch, cs, cc, bd, bt);
-                // advance the carry over the cells of the buckets just processed
-                uint32_t part = 0, ptot;
-                for (int cidx = kstart * cpb + tid; cidx < k * cpb; cidx += nt) part = max(part, cmx[cidx]);
-                block_scan_excl<uint32_t>(part, OpMax(), 0u, (uint32_t *)tmp, &ptot);
-                carry_batch = max(carry_batch, ptot);
-                kstart = k;
+                carry_batch = g0[(size_t)k * cpb];        // G at the start of the next batch's first bucket
                 m = 0;
             }
             const uint64_t *src = list + (size_t)k * F.capb;
@@ -814,6 +842,34 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
         if (m > 0) run_batch<uint32_t, ZL_OBJ_RANGE>(keys, m, (uint32_t)M.t0, n, tmp, carry_batch, cs, cc, bd, bt);
     }
     block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres + g]);
+}
+
+// Instances with few survivors of the filter pass: one CTA gathers the regions' lists, sorts them and
+// sweeps them, with nothing before them to carry in.
+__global__ void __launch_bounds__(1024) k_tail(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg) {
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ uint64_t tmp[34];
+    __shared__ unsigned int sstatus, fill;
+    const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+    const InstMeta M = meta[b];
+    if (M.status != ZL_OK || !handled_by_filter(M, 1) || !tail_instance(M)) return;
+    Key<uint32_t> *keys = (Key<uint32_t> *)smem;
+    if (tid == 0) { sstatus = 0; fill = 0; }
+    __syncthreads();
+    for (int r = warp; r < F.nreg; r += nw) {
+        const uint32_t c = F.rcnt[(size_t)b * F.nreg + r];
+        if (c == 0) continue;
+        uint32_t off = 0;
+        if (lane == 0) off = atomicAdd(&fill, c);
+        off = __shfl_sync(FULL, off, 0);
+        const uint64_t *src = F.list1 + (size_t)b * F.list1cap + (size_t)r * F.regcap;
+        for (uint32_t i = lane; i < c; i += 32) keys[off + i].w = src[i];
+    }
+    __syncthreads();
+    uint64_t bd = ~0ull, bt = ~0ull, cs = 0;
+    uint32_t cc = 0;
+    run_batch<uint32_t, ZL_OBJ_RANGE>(keys, (int)M.count, (uint32_t)M.t0, n, tmp, (uint32_t)0, cs, cc, bd, bt);
+    block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres]);
 }
 
 // ------------------------------------------------------------------------------ finalize
@@ -832,7 +888,7 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
     uint64_t bd = ~0ull, bt = ~0ull;
     uint32_t st = M.status;
     if (st == ZL_OK) {
-        const int used = handled_by_filter(M, filter) ? (F.nbk + bucket_group(F, M.count2) - 1) / bucket_group(F, M.count2) : nseg;
+        const int used = !handled_by_filter(M, filter) ? nseg : tail_instance(M) ? 1 : (F.nbk + bucket_group(F, M.count2) - 1) / bucket_group(F, M.count2);
         for (int s = tid; s < used; s += blockDim.x) {
             const SegResult r = seg[(size_t)b * nres + s];
             if (r.status != ZL_OK) st = max(st, (uint32_t)r.status);
@@ -854,15 +910,38 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
         barrier[b] = bar;
         if (status) status[b] = fst;
     }
+    // one thread per row: the number of elements <= barrier.  Rows are close to arithmetic, so the position is
+    // first guessed from the row's end points, bracketed by doubling steps around the guess, then bisected.
     const int p = blockIdx.x * blockDim.x + tid;
     if (p < n) {
         int res = -1;
         if (fst == ZL_OK) {
             const int64_t *row = ts + ((size_t)b * n + p) * R;
-            int lo = 0, hi = R;                   // number of elements <= barrier
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if (ldg64(row + mid) <= bar) lo = mid + 1; else hi = mid;
+            const int64_t e0 = ldg64(row), eR = ldg64(row + R - 1);
+            int lo, hi;                           // invariant: row[lo - 1] <= bar (or lo == 0), row[hi] > bar (or hi == R)
+            if (bar < e0) { lo = 0; hi = 0; }
+            else if (bar >= eR) { lo = R; hi = R; }
+            else {
+                // e0 <= bar < eR, R >= 2
+                int g = (int)((double)(bar - e0) * (double)(R - 1) / (double)(eR - e0));
+                g = max(0, min(g, R - 2));
+                if (ldg64(row + g) <= bar) {
+                    lo = g + 1; hi = R - 1;       // row[R-1] > bar
+                    for (int step = 1; lo < hi; step <<= 1) {
+                        const int q = min(lo + step - 1, hi - 1);
+                        if (ldg64(row + q) <= bar) lo = q + 1; else { hi = q; break; }
+                    }
+                } else {
+                    hi = g; lo = 1;               // row[0] <= bar
+                    for (int step = 1; lo < hi; step <<= 1) {
+                        const int q = max(hi - step, lo);
+                        if (ldg64(row + q) > bar) hi = q; else { lo = q + 1; break; }
+                    }
+                }
+                while (lo < hi) {
+                    const int mid = (lo + hi) >> 1;
+                    if (ldg64(row + mid) <= bar) lo = mid + 1; else hi = mid;
+                }
             }
             res = lo - 1;
         }
@@ -963,7 +1042,7 @@ struct zl_handle {
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows;
     int last_cuda_error;
     int launches;
     // optional per-kernel timing: PROF_EVENTS events per recorded call
@@ -984,6 +1063,7 @@ struct Pipeline {
     const int64_t *ts; int B, n, R, objective, flags, num_sms;
     zl::InstMeta *meta; zl::SegResult *seg; int nres;
     zl::FilterBufs fb;                                            // fb.table == nullptr: no filter route
+    int filter_threads, filter_rows;                              // 0: automatic
     int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;
 };
 
@@ -1001,17 +1081,21 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     }
     if (ev) cudaEventRecord(ev[1], st);
     if (filter) {
-        const int threads = std::max(64, std::min(1024, 32 * pow2_ceil(std::min(q.n, 32))));
+        int threads = std::max(64, std::min(256, 32 * pow2_ceil(std::min(q.n, 32))));
+        if (q.filter_threads) threads = std::max(64, std::min(q.filter_threads, 32 * pow2_ceil(std::min(q.n, 32))));
         const int nw = threads / 32;
-        long long rpc = ((long long)q.n * q.B / (4LL * q.num_sms) + nw - 1) / nw * nw;
+        long long rpc = ((long long)q.n * q.B / (16LL * q.num_sms) + nw - 1) / nw * nw;
+        if (q.filter_rows) rpc = ((long long)q.filter_rows + nw - 1) / nw * nw;
         rpc = std::max<long long>(nw, std::min<long long>(rpc, (q.n + nw - 1) / nw * nw));
         fb.nreg = (int)((q.n + rpc - 1) / rpc);
         fb.regcap = fb.list1cap / fb.nreg;
         const size_t fsmem = (size_t)fb.cells * 4 + (size_t)nw * zl::FILTER_STAGES * zl::FILTER_SLOT * 8;
         zl::k_filter<<<dim3(fb.nreg, q.B), threads, fsmem, st>>>(q.ts, q.n, q.R, q.flags, (int)rpc, q.meta, fb);
         if (ev) cudaEventRecord(ev[2], st);
-        const int rthreads = std::max(128, std::min(1024, fb.cells / 4));
-        zl::k_refine<<<dim3(fb.nreg, q.B), rthreads, (size_t)fb.cells * 4, st>>>(q.meta, fb);
+        const int tcap = (int)std::min<long long>((long long)zl::TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
+        zl::k_tail<<<q.B, std::max(64, std::min(1024, tcap / 4)), (size_t)tcap * 8, st>>>(q.meta, fb, q.n, q.nres, q.seg);
+        zl::k_cellscan<<<q.B, std::max(64, std::min(1024, fb.fcells / 4)), 0, st>>>(q.meta, fb);
+        zl::k_refine<<<dim3(fb.nreg, q.B), std::max(64, std::min(1024, pow2_ceil(fb.regcap / 4))), 0, st>>>(q.meta, fb);
         const int ngroups = (fb.nbk + fb.grp - 1) / fb.grp;
         const int bthreads = std::max(64, std::min(256, fb.capb / 4));
         zl::k_buckets<<<dim3(ngroups, q.B), bthreads, (size_t)fb.capb * 8, st>>>(q.meta, fb, q.n, q.nres, q.seg);
@@ -1028,7 +1112,8 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     if (q.objective == ZL_OBJ_RANGE) zl::k_sweep<ZL_OBJ_RANGE><<<sweep_ctas, p.threads, p.smem, st>>>(sp);
     else zl::k_sweep<ZL_OBJ_SUM><<<sweep_ctas, p.threads, p.smem, st>>>(sp);
     if (ev) cudaEventRecord(ev[3], st);
-    zl::k_finalize<<<dim3((q.n + 255) / 256, q.B), 256, 0, st>>>(q.ts, q.n, q.R, p.nseg, fb, q.nres, q.objective,
+    const int fthreads = std::max(32, std::min(256, pow2_ceil(q.n)));
+    zl::k_finalize<<<dim3((q.n + fthreads - 1) / fthreads, q.B), fthreads, 0, st>>>(q.ts, q.n, q.R, p.nseg, fb, q.nres, q.objective,
                                                                   filter ? 1 : 0, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
     if (ev) cudaEventRecord(ev[4], st);
 }
@@ -1038,7 +1123,7 @@ cudaError_t raise_shared_memory_limits() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_buckets, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_refine, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_tail, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     return e;
 }
 
@@ -1124,13 +1209,14 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         const long long N = (long long)cfg->n_workers * cfg->lookahead_R;
         const size_t mb = (size_t)cfg->max_batch;
         zl::FilterBufs &f = h->fb;
-        f.cells = std::max(64, std::min(zl::FILTER_MAX_CELLS, pow2_ceil((int)std::min<long long>(4LL * cfg->lookahead_R, 1 << 20))));
+        f.cells = std::max(64, std::min(zl::FILTER_MAX_CELLS, pow2_ceil((int)std::min<long long>(cfg->lookahead_R, 1 << 20))));
         f.capb = (int)std::max<long long>(64, std::min<long long>(4096, pow2_ceil((int)std::min<long long>(N, 1 << 20))));
-        f.nbk = (int)std::max<long long>(1, std::min<long long>(std::min(1024, f.cells), pow2_ceil((int)std::min<long long>(N / 8 / f.capb, 1 << 20))));
+        f.nbk = (int)std::max<long long>(1, std::min<long long>(1024, pow2_ceil((int)std::min<long long>(N / 8 / f.capb, 1 << 20))));
+        f.fcells = (int)std::max<long long>(std::max(64, f.nbk), std::min<long long>(1 << 18, pow2_ceil((int)std::min<long long>(N / 64, 1 << 20))));
         f.grp = std::max(1, std::min(f.nbk, pow2_floor((int)std::max<long long>(1, (long long)f.nbk * cfg->max_batch / (8LL * std::max(1, h->num_sms))))));
         f.list1cap = (int)std::max<long long>(N / 2, std::min<long long>(N, 4096));
         h->nres = std::max(zl::MAX_SEGMENTS, (f.nbk + f.grp - 1) / f.grp);
-        const size_t sizes[7] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.cells * 4, mb * cfg->n_workers * 4,
+        const size_t sizes[7] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.fcells * 4, mb * cfg->n_workers * 4,
                                  mb * (size_t)f.list1cap * 8, mb * f.nbk * 4, mb * f.nbk * f.capb * 8};
         void **ptrs[7] = {(void **)&f.table, (void **)&f.rowhint, (void **)&f.cellmax, (void **)&f.rcnt,
                           (void **)&f.list1, (void **)&f.bcnt, (void **)&f.list2};
@@ -1231,6 +1317,12 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
         h->opt_segments = value;
     } else if (!strcmp(key, "no_filter")) {
         h->opt_no_filter = value != 0;
+    } else if (!strcmp(key, "filter_threads")) {
+        if (value && (!is_pow2(value) || value < 64 || value > 1024)) return ZL_ERR_INVALID_ARG;
+        h->opt_filter_threads = value;
+    } else if (!strcmp(key, "filter_rows")) {
+        if (value > 65536) return ZL_ERR_INVALID_ARG;
+        h->opt_filter_rows = value;
     } else if (!strcmp(key, "round_factor")) {
         if (value > 100000) return ZL_ERR_INVALID_ARG;
         h->opt_round_factor = value;
@@ -1244,7 +1336,7 @@ size_t zl_workspace_bytes(const zl_handle *h) { return h ? h->ws_bytes + h->stag
 int32_t zl_launches_per_call(const zl_handle *h) {
     if (!h) return 0;
     const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter;
-    return 3 + (filter ? 3 : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
+    return 3 + (filter ? 5 : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
 }
 int32_t zl_segments_per_instance(const zl_handle *h, int32_t B) { return h && B >= 1 ? make_plan(h, B).nseg : 0; }
 int32_t zl_last_cuda_error(const zl_handle *h) { return h ? h->last_cuda_error : 0; }
@@ -1266,6 +1358,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.ts = d_ts; q.B = B; q.n = n; q.R = R; q.objective = obj; q.flags = h->cfg.flags; q.num_sms = h->num_sms;
     q.meta = h->d_meta; q.seg = h->d_seg; q.nres = h->nres;
     q.fb = h->fb;
+    q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows;
     if (h->opt_no_filter) q.fb.table = nullptr;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, st, ev);
@@ -1406,6 +1499,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
     q.meta = meta; q.seg = seg; q.nres = p.nseg;
     memset(&q.fb, 0, sizeof(q.fb));
+    q.filter_threads = q.filter_rows = 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr);
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;
