@@ -43,7 +43,7 @@ struct InstMeta {
     uint32_t count;      // survivors of the filter pass
     uint32_t count2;     // survivors of the refinement
     uint32_t overflow;   // a survivor list overflowed: the instance takes the segment sweep instead
-    uint32_t pad;
+    uint32_t dmin;       // no element whose own iteration (next - T) is this short can pass the filter table
 };
 
 struct SegResult {
@@ -61,8 +61,10 @@ struct FilterBufs {
     uint32_t *rowhint;   // [B][n]            estimated number of elements of a row that are <= lmin
     uint32_t *cellmax;   // [B][fcells]       max `next` over the filter pass's survivors of each fine cell; after
                          //                   k_cellscan: G at the start of each fine cell
+    uint32_t *tilemax;   // [B][fcells/4096]  max of cellmax per tile of 4096 fine cells (scratch of the cell scan)
     uint32_t *rcnt;      // [B][nreg]         survivors per region (one region per CTA of the filter pass)
     uint64_t *list1;     // [B][list1cap]     survivors of the filter pass as (T << 32 | next), by region
+    uint32_t *flags;     // [2]               per call: [0] some instance needs scan/refine/buckets, [1] some needs the segment sweep
     uint32_t *bcnt;      // [B][nbk]          survivors of the refinement per bucket
     uint64_t *list2;     // [B][nbk][capb]    survivors of the refinement
     int32_t cells, fcells, nbk, capb, grp;   // grp: fewest buckets per CTA of the bucket sweep
@@ -75,6 +77,7 @@ struct SweepParams {
     SegResult *seg;
     int32_t n, R, B, nseg, nres, G, cap, flags, target;   // nres: SegResult slots per instance
     int32_t filter;      // instances handled by the filter route are skipped
+    const uint32_t *need; // filter on: [1] != 0 when some instance needs this sweep; nullptr: always run
 };
 
 // Buckets per CTA of the bucket sweep for an instance with `count` refined survivors: the static
@@ -139,7 +142,7 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
         InstMeta m;
         m.tmin = tmin;
         m.status = ZL_OK;
-        m.cscale = 0; m.fscale = 0; m.count = 0; m.count2 = 0; m.overflow = 0; m.pad = 0;
+        m.cscale = 0; m.fscale = 0; m.count = 0; m.count2 = 0; m.overflow = 0; m.dmin = 0;
         if (tmin < 0 || tmax >= VALUE_LIMIT || tmax < tmin || lmin < tmin) {
             m.status = ZL_ERR_INVALID_ARG;     // outside [0, 2^62), or first/last columns out of order
             m.t0 = m.lmin = m.tend = 1; m.use32 = 1;
@@ -159,8 +162,10 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
     }
     __syncthreads();
     const InstMeta M = sm;
+    if (b == 0 && tid < 2 && F.flags) F.flags[tid] = 0;
     if (M.cscale != 0) {
         const uint32_t cells = (uint32_t)F.cells, cscale = M.cscale, lmin = (uint32_t)M.lmin;
+        const uint32_t wcell = 0xffffffffu / cscale + 2;          // > 2^32 / cscale
         const int64_t tmin = M.tmin;
         uint32_t *cmx = F.cellmax + (size_t)b * F.fcells;
         for (uint32_t c = tid; c < cells; c += nt) tab[c] = (uint32_t)M.t0;
@@ -220,9 +225,28 @@ __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int
         }
         __syncthreads();
         uint32_t *tg = F.table + (size_t)b * cells;
-        for (uint32_t c = tid; c < cells; c += nt) tg[c] = tab[c];
+        // dmin: every T of cell c is <= tmax_c, so an element with next - T <= tab[c] - tmax_c for all c never passes
+        uint32_t dloc = 0xffffffffu;
+        for (uint32_t c = tid; c < cells; c += nt) {
+            const uint32_t v = tab[c];
+            tg[c] = v;
+            // upper bound of the times of cell c: a cell spans fewer than wcell time units
+            const uint64_t tmax_c = min((uint64_t)lmin, (uint64_t)(c + 1) * wcell + 1);
+            dloc = min(dloc, (uint64_t)v > tmax_c ? (uint32_t)(v - tmax_c) : 0u);
+        }
+        dloc = warp_reduce(dloc, OpMin());
+        __syncthreads();
+        uint32_t *red = (uint32_t *)&s[0][0];
+        if (lane == 0) red[warp] = dloc;
+        __syncthreads();
+        if (tid == 0) {
+            uint32_t d = 0xffffffffu;
+            for (int w = 0; w < nw; ++w) d = min(d, red[w]);
+            sm.dmin = d;
+        }
+        __syncthreads();
     }
-    if (tid == 0) meta[b] = M;
+    if (tid == 0) meta[b] = sm;
     (void)flags;
 }
 
@@ -259,16 +283,18 @@ __device__ __forceinline__ void cp_async_wait_pending(int pending) {
 
 struct FilterCtx {
     const uint32_t *tab; uint64_t *list; uint32_t *cellmax; unsigned int *scount;
-    uint32_t cscale, fscale, lmin, regcap;
+    uint32_t cscale, fscale, lmin, regcap, dmin;
 };
 
 // Table test of the (up to) two elements of a lane, warp-aggregated append of the survivors.
 __device__ __forceinline__ void filter_pair(const FilterCtx &c, int lane, bool va, uint32_t Ta, uint32_t na,
                                             bool vb, uint32_t Tb, uint32_t nb) {
-    bool ka = false, kb = false;
-    uint32_t ca = 0, cb = 0;
-    if (va && Ta <= c.lmin) { ca = cell_of(Ta, c.cscale); ka = na > max(Ta, c.tab[ca]); }
-    if (vb && Tb <= c.lmin) { cb = cell_of(Tb, c.cscale); kb = nb > max(Tb, c.tab[cb]); }
+    // cheap necessary condition first: most elements belong to fast workers and stop here
+    bool ka = va && Ta <= c.lmin && na - Ta > c.dmin;
+    bool kb = vb && Tb <= c.lmin && nb - Tb > c.dmin;
+    if (!__any_sync(FULL, ka || kb)) return;
+    if (ka) ka = na > max(Ta, c.tab[cell_of(Ta, c.cscale)]);
+    if (kb) kb = nb > max(Tb, c.tab[cell_of(Tb, c.cscale)]);
     const unsigned ma = __ballot_sync(FULL, ka), mb = __ballot_sync(FULL, kb);
     if ((ma | mb) == 0) return;
     const int na_cnt = __popc(ma), tot = na_cnt + __popc(mb);
@@ -323,7 +349,7 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
     FilterCtx C;
     C.tab = tab; C.list = F.list1 + (size_t)b * F.list1cap + (size_t)blockIdx.x * F.regcap;
     C.cellmax = F.cellmax + (size_t)b * F.fcells; C.scount = &scount;
-    C.cscale = M.cscale; C.fscale = M.fscale; C.lmin = lmin; C.regcap = (uint32_t)F.regcap;
+    C.cscale = M.cscale; C.fscale = M.fscale; C.lmin = lmin; C.regcap = (uint32_t)F.regcap; C.dmin = M.dmin;
     const int r0 = blockIdx.x * rows_per_cta, r1 = min(r0 + rows_per_cta, n);
     const bool vec2 = (R % 2 == 0) && (((uintptr_t)ts & 15) == 0);
     const int nchunks = (R + FILTER_CHUNK - 1) / FILTER_CHUNK;
@@ -407,18 +433,49 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
 // every element that ever raises the running maximum): k_cellscan turns cellmax, in place, into its
 // exclusive prefix maximum floored by t0.  A survivor whose `next` does not exceed G at the start of its
 // own cell cannot matter either, so k_refine drops it; the rest go to their time bucket.
-__global__ void __launch_bounds__(1024) k_cellscan(const InstMeta *meta, FilterBufs F) {
+constexpr int SCAN_TILE = 4096;
+
+// pass 1: maximum of every tile of SCAN_TILE fine cells.  A fixed grid walks the (tile, instance) pairs.
+__global__ void __launch_bounds__(256) k_tilemax(const InstMeta *meta, FilterBufs F, int B) {
     __shared__ uint64_t tmp[34];
-    __shared__ uint32_t tile[4096];
-    const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
-    const InstMeta M = meta[b];
-    if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) return;
-    uint32_t *cmx = F.cellmax + (size_t)b * F.fcells;
-    uint32_t carry = (uint32_t)M.t0;
-    // tiles of 4096 cells: coalesced in, each thread scans a run of consecutive cells, coalesced out
-    for (int base = 0; base < F.fcells; base += 4096) {
-        const int len = min(4096, F.fcells - base);
-        for (int i = tid; i < len; i += nt) tile[i] = cmx[base + i];
+    if (F.flags[0] == 0) return;                                  // no instance takes this route in this call
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int tiles = (F.fcells + SCAN_TILE - 1) / SCAN_TILE;
+    for (int item = blockIdx.x; item < tiles * B; item += gridDim.x) {
+        const int b = item / tiles, t = item % tiles;
+        const InstMeta M = meta[b];
+        if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) continue;
+        const uint32_t *cmx = F.cellmax + (size_t)b * F.fcells + (size_t)t * SCAN_TILE;
+        const int len = min(SCAN_TILE, F.fcells - t * SCAN_TILE);
+        uint32_t loc = 0;
+        for (int i = tid; i < len; i += nt) loc = max(loc, cmx[i]);
+        uint32_t tot;
+        block_scan_excl<uint32_t>(loc, OpMax(), 0u, (uint32_t *)tmp, &tot);
+        if (tid == 0) F.tilemax[(size_t)b * tiles + t] = tot;
+    }
+}
+
+// pass 2: each tile becomes, in place, the exclusive prefix maximum over all cells before each of its
+// cells, floored by t0: coalesced in, every thread scans a run of consecutive cells in shared memory,
+// coalesced out.
+__global__ void __launch_bounds__(256) k_cellscan(const InstMeta *meta, FilterBufs F, int B) {
+    __shared__ uint64_t tmp[34];
+    __shared__ uint32_t tile[SCAN_TILE];
+    if (F.flags[0] == 0) return;
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int tiles = (F.fcells + SCAN_TILE - 1) / SCAN_TILE;
+    for (int item = blockIdx.x; item < tiles * B; item += gridDim.x) {
+        const int b = item / tiles, t = item % tiles;
+        const InstMeta M = meta[b];
+        if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) continue;
+        uint32_t *cmx = F.cellmax + (size_t)b * F.fcells + (size_t)t * SCAN_TILE;
+        const int len = min(SCAN_TILE, F.fcells - t * SCAN_TILE);
+        uint32_t before = 0;
+        for (int i = tid; i < t; i += nt) before = max(before, F.tilemax[(size_t)b * tiles + i]);
+        uint32_t carry;
+        block_scan_excl<uint32_t>(before, OpMax(), 0u, (uint32_t *)tmp, &carry);
+        carry = max(carry, (uint32_t)M.t0);
+        for (int i = tid; i < len; i += nt) tile[i] = cmx[i];
         __syncthreads();
         const int per = (len + nt - 1) / nt;
         const int c0 = min(tid * per, len), c1 = min(c0 + per, len);
@@ -427,40 +484,54 @@ __global__ void __launch_bounds__(1024) k_cellscan(const InstMeta *meta, FilterB
         uint32_t tot;
         uint32_t run = max(block_scan_excl<uint32_t>(loc, OpMax(), 0u, (uint32_t *)tmp, &tot), carry);
         for (int c = c0; c < c1; ++c) { const uint32_t v = tile[c]; tile[c] = run; run = max(run, v); }
-        carry = max(carry, tot);
         __syncthreads();
-        for (int i = tid; i < len; i += nt) cmx[base + i] = tile[i];
+        for (int i = tid; i < len; i += nt) cmx[i] = tile[i];
         __syncthreads();
     }
 }
 
-__global__ void __launch_bounds__(1024) k_refine(InstMeta *meta, FilterBufs F) {
-    const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
-    const InstMeta M = meta[b];
-    if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) return;
-    const uint32_t m = F.rcnt[(size_t)b * F.nreg + blockIdx.x];
-    if (m == 0) return;
-    const uint32_t *g = F.cellmax + (size_t)b * F.fcells;         // G at fine cell starts
-    const uint64_t *src = F.list1 + (size_t)b * F.list1cap + (size_t)blockIdx.x * F.regcap;
-    uint32_t *bcnt = F.bcnt + (size_t)b * F.nbk;
-    uint64_t *dst = F.list2 + (size_t)b * F.nbk * F.capb;
+__global__ void __launch_bounds__(256) k_refine(InstMeta *meta, FilterBufs F, int B) {
+    if (F.flags[0] == 0) return;
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
     const int cpb_shift = __ffs(F.fcells / F.nbk) - 1;            // fine cells per bucket is a power of two
-    unsigned kept = 0;
-    bool over = false;
-    for (uint32_t i = tid; i < m; i += nt) {
-        const uint64_t w = src[i];
-        const uint32_t T = (uint32_t)(w >> 32), nx = (uint32_t)w;
-        const uint32_t c = cell_of(T, M.fscale);
-        if (nx > max(T, __ldg(g + c))) {
-            const uint32_t bk = c >> cpb_shift;
-            const uint32_t pos = atomicAdd(&bcnt[bk], 1u);
-            if (pos < (uint32_t)F.capb) dst[(size_t)bk * F.capb + pos] = w; else over = true;
-            ++kept;
+    for (int item = blockIdx.x; item < F.nreg * B; item += gridDim.x) {
+        const int b = item / F.nreg, reg = item % F.nreg;
+        const InstMeta M = meta[b];
+        if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) continue;
+        const uint32_t m = F.rcnt[(size_t)b * F.nreg + reg];
+        if (m == 0) continue;
+        const uint32_t *g = F.cellmax + (size_t)b * F.fcells;     // G at fine cell starts
+        const uint64_t *src = F.list1 + (size_t)b * F.list1cap + (size_t)reg * F.regcap;
+        uint32_t *bcnt = F.bcnt + (size_t)b * F.nbk;
+        uint64_t *dst = F.list2 + (size_t)b * F.nbk * F.capb;
+        unsigned kept = 0;
+        bool over = false;
+        // four elements a step, so that four list loads and then four table look-ups are in flight together
+        for (uint32_t i0 = tid; i0 < m; i0 += 4 * nt) {
+            uint64_t w[4];
+            uint32_t c[4], gv[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { const uint32_t i = i0 + k * nt; w[k] = i < m ? src[i] : 0ull; }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                c[k] = w[k] ? cell_of((uint32_t)(w[k] >> 32), M.fscale) : 0u;
+                gv[k] = __ldg(g + c[k]);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t T = (uint32_t)(w[k] >> 32), nx = (uint32_t)w[k];
+                if (w[k] && nx > max(T, gv[k])) {
+                    const uint32_t bk = c[k] >> cpb_shift;
+                    const uint32_t pos = atomicAdd(&bcnt[bk], 1u);
+                    if (pos < (uint32_t)F.capb) dst[(size_t)bk * F.capb + pos] = w[k]; else over = true;
+                    ++kept;
+                }
+            }
         }
+        kept = warp_reduce(kept, OpAdd());
+        if (lane == 0 && kept) atomicAdd(&meta[b].count2, kept);
+        if (over) { meta[b].overflow = 1; F.flags[1] = 1; }
     }
-    kept = warp_reduce(kept, OpAdd());
-    if (lane == 0 && kept) atomicAdd(&meta[b].count2, kept);
-    if (over) meta[b].overflow = 1;
 }
 
 // Optional full check that every row is non-decreasing.
@@ -758,6 +829,7 @@ __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
     uint32_t *curA = (uint32_t *)smem;
     uint32_t *curB = curA + P.n;
     unsigned char *kb = smem + (((size_t)2 * P.n * sizeof(uint32_t) + 15) & ~(size_t)15);
+    if (P.need && P.need[1] == 0) return;                        // the filter route finished every instance
     // a fixed number of CTAs walks the (instance, segment) pairs
     const int items = P.B * P.nseg;
     for (int item = blockIdx.x; item < items; item += gridDim.x) {
@@ -784,19 +856,24 @@ __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
 // Sort and sweep the refined survivors.  CTA (g, b) takes buckets [g*grp, (g+1)*grp) of instance b in
 // time order, packs whole buckets into shared-memory batches and runs each batch with the running
 // maximum of `next` over everything before it (the prefix maximum of cellmax up to the batch's first cell).
-__global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg) {
+__global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg, int B) {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
     __shared__ unsigned int sstatus, fill;
-    const int b = blockIdx.y, g = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
-    const InstMeta M = meta[b];
-    if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) return;
+    if (F.flags[0] == 0) return;                                  // no instance takes this route in this call
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int ngroups = (F.nbk + F.grp - 1) / F.grp;
     Key<uint32_t> *keys = (Key<uint32_t> *)smem;
+    for (int item = blockIdx.x; item < ngroups * B; item += gridDim.x) {
+    const int b = item / ngroups, g = item % ngroups;
+    __syncthreads();                                              // shared state of the previous item is done with
+    const InstMeta M = meta[b];
+    if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) continue;
     const uint32_t *bcnt = F.bcnt + (size_t)b * F.nbk;
     const uint32_t *g0 = F.cellmax + (size_t)b * F.fcells;        // G at fine cell starts (after k_cellscan)
     const uint64_t *list = F.list2 + (size_t)b * F.nbk * F.capb;
     const int grp = bucket_group(F, M.count2);
-    if (g * grp >= F.nbk) return;                                // fewer, wider groups than CTAs for this instance
+    if (g * grp >= F.nbk) continue;                              // fewer, wider groups than items for this instance
     const int first = g * grp, last = min(first + grp, F.nbk);
     const int cpb = F.fcells / F.nbk;
     if (tid == 0) { sstatus = 0; fill = 0; }
@@ -842,33 +919,71 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
         if (m > 0) run_batch<uint32_t, ZL_OBJ_RANGE>(keys, m, (uint32_t)M.t0, n, tmp, carry_batch, cs, cc, bd, bt);
     }
     block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres + g]);
+    }
 }
 
-// Instances with few survivors of the filter pass: one CTA gathers the regions' lists, sorts them and
-// sweeps them, with nothing before them to carry in.
+// Instances with few survivors of the filter pass are finished by one CTA.  It first applies the
+// refinement at the resolution of the coarse cells, in shared memory (maximum of next per cell,
+// exclusive prefix maximum, drop every survivor whose next does not exceed the value at its cell's
+// start), then sorts what is left and sweeps it.  Dropped survivors never hold the running maximum
+// alone, so nothing has to be carried in.
 __global__ void __launch_bounds__(1024) k_tail(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg) {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
     __shared__ unsigned int sstatus, fill;
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
     const InstMeta M = meta[b];
+    if (M.status == ZL_OK && tid == 0) {
+        // tell the later kernels of this call whether they have anything to do
+        if (!handled_by_filter(M, 1)) F.flags[1] = 1;
+        else if (!tail_instance(M)) F.flags[0] = 1;
+    }
     if (M.status != ZL_OK || !handled_by_filter(M, 1) || !tail_instance(M)) return;
-    Key<uint32_t> *keys = (Key<uint32_t> *)smem;
+    uint32_t *g = (uint32_t *)smem;                               // [cells]
+    Key<uint32_t> *keys = (Key<uint32_t> *)(smem + (size_t)F.cells * 4);
+    const int cells = F.cells;
+    for (int c = tid; c < cells; c += nt) g[c] = 0;
     if (tid == 0) { sstatus = 0; fill = 0; }
     __syncthreads();
     for (int r = warp; r < F.nreg; r += nw) {
         const uint32_t c = F.rcnt[(size_t)b * F.nreg + r];
-        if (c == 0) continue;
-        uint32_t off = 0;
-        if (lane == 0) off = atomicAdd(&fill, c);
-        off = __shfl_sync(FULL, off, 0);
         const uint64_t *src = F.list1 + (size_t)b * F.list1cap + (size_t)r * F.regcap;
-        for (uint32_t i = lane; i < c; i += 32) keys[off + i].w = src[i];
+        for (uint32_t i = lane; i < c; i += 32) {
+            const uint64_t w = src[i];
+            atomicMax(&g[cell_of((uint32_t)(w >> 32), M.cscale)], (uint32_t)w);
+        }
+    }
+    __syncthreads();
+    {   // exclusive prefix maximum over the cells, floored by t0
+        const int per = (cells + nt - 1) / nt;
+        const int c0 = min(tid * per, cells), c1 = min(c0 + per, cells);
+        uint32_t loc = 0;
+        for (int c = c0; c < c1; ++c) loc = max(loc, g[c]);
+        uint32_t tot;
+        uint32_t run = max(block_scan_excl<uint32_t>(loc, OpMax(), 0u, (uint32_t *)tmp, &tot), (uint32_t)M.t0);
+        for (int c = c0; c < c1; ++c) { const uint32_t v = g[c]; g[c] = run; run = max(run, v); }
+    }
+    __syncthreads();
+    for (int r = warp; r < F.nreg; r += nw) {
+        const uint32_t c = F.rcnt[(size_t)b * F.nreg + r];
+        const uint64_t *src = F.list1 + (size_t)b * F.list1cap + (size_t)r * F.regcap;
+        for (uint32_t i0 = 0; i0 < c; i0 += 32) {
+            const uint32_t i = i0 + lane;
+            const uint64_t w = i < c ? src[i] : 0ull;
+            const uint32_t T = (uint32_t)(w >> 32), nx = (uint32_t)w;
+            const bool keep = i < c && nx > max(T, g[cell_of(T, M.cscale)]);
+            const unsigned km = __ballot_sync(FULL, keep);
+            if (km == 0) continue;
+            unsigned base = 0;
+            if (lane == 0) base = atomicAdd(&fill, (unsigned)__popc(km));
+            base = __shfl_sync(FULL, base, 0);
+            if (keep) keys[base + __popc(km & ((1u << lane) - 1u))].w = w;
+        }
     }
     __syncthreads();
     uint64_t bd = ~0ull, bt = ~0ull, cs = 0;
     uint32_t cc = 0;
-    run_batch<uint32_t, ZL_OBJ_RANGE>(keys, (int)M.count, (uint32_t)M.t0, n, tmp, (uint32_t)0, cs, cc, bd, bt);
+    run_batch<uint32_t, ZL_OBJ_RANGE>(keys, (int)fill, (uint32_t)M.t0, n, tmp, (uint32_t)0, cs, cc, bd, bt);
     block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres]);
 }
 
@@ -1093,12 +1208,16 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         zl::k_filter<<<dim3(fb.nreg, q.B), threads, fsmem, st>>>(q.ts, q.n, q.R, q.flags, (int)rpc, q.meta, fb);
         if (ev) cudaEventRecord(ev[2], st);
         const int tcap = (int)std::min<long long>((long long)zl::TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
-        zl::k_tail<<<q.B, std::max(64, std::min(1024, tcap / 4)), (size_t)tcap * 8, st>>>(q.meta, fb, q.n, q.nres, q.seg);
-        zl::k_cellscan<<<q.B, std::max(64, std::min(1024, fb.fcells / 4)), 0, st>>>(q.meta, fb);
-        zl::k_refine<<<dim3(fb.nreg, q.B), std::max(64, std::min(1024, pow2_ceil(fb.regcap / 4))), 0, st>>>(q.meta, fb);
+        zl::k_tail<<<q.B, std::max(64, std::min(1024, tcap / 2)), (size_t)tcap * 8 + (size_t)fb.cells * 4, st>>>(q.meta, fb, q.n, q.nres, q.seg);
+        // the route for instances with many survivors: fixed-size grids that return at once when no instance needs them
+        const int tiles = (fb.fcells + zl::SCAN_TILE - 1) / zl::SCAN_TILE;
+        const int wide = 4 * q.num_sms;
+        zl::k_tilemax<<<std::min(tiles * q.B, wide), 256, 0, st>>>(q.meta, fb, q.B);
+        zl::k_cellscan<<<std::min(tiles * q.B, wide), 256, 0, st>>>(q.meta, fb, q.B);
+        zl::k_refine<<<std::min(fb.nreg * q.B, wide), 256, 0, st>>>(q.meta, fb, q.B);
         const int ngroups = (fb.nbk + fb.grp - 1) / fb.grp;
         const int bthreads = std::max(64, std::min(256, fb.capb / 4));
-        zl::k_buckets<<<dim3(ngroups, q.B), bthreads, (size_t)fb.capb * 8, st>>>(q.meta, fb, q.n, q.nres, q.seg);
+        zl::k_buckets<<<std::min(ngroups * q.B, wide), bthreads, (size_t)fb.capb * 8, st>>>(q.meta, fb, q.n, q.nres, q.seg, q.B);
     } else if (ev) {
         cudaEventRecord(ev[2], st);
     }
@@ -1106,6 +1225,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     sp.ts = q.ts; sp.meta = q.meta; sp.seg = q.seg;
     sp.n = q.n; sp.R = q.R; sp.B = q.B; sp.nseg = p.nseg; sp.nres = q.nres; sp.G = p.G; sp.cap = p.cap;
     sp.flags = q.flags; sp.target = p.target; sp.filter = filter ? 1 : 0;
+    sp.need = filter ? fb.flags : nullptr;
     // with the filter route on, the segment sweep is only the fallback: a small persistent grid
     const int items = p.nseg * q.B;
     const int sweep_ctas = filter ? std::min(items, 2 * q.num_sms) : items;
@@ -1216,11 +1336,12 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         f.grp = std::max(1, std::min(f.nbk, pow2_floor((int)std::max<long long>(1, (long long)f.nbk * cfg->max_batch / (8LL * std::max(1, h->num_sms))))));
         f.list1cap = (int)std::max<long long>(N / 2, std::min<long long>(N, 4096));
         h->nres = std::max(zl::MAX_SEGMENTS, (f.nbk + f.grp - 1) / f.grp);
-        const size_t sizes[7] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.fcells * 4, mb * cfg->n_workers * 4,
-                                 mb * (size_t)f.list1cap * 8, mb * f.nbk * 4, mb * f.nbk * f.capb * 8};
-        void **ptrs[7] = {(void **)&f.table, (void **)&f.rowhint, (void **)&f.cellmax, (void **)&f.rcnt,
-                          (void **)&f.list1, (void **)&f.bcnt, (void **)&f.list2};
-        for (int i = 0; i < 7; ++i) {
+        const size_t tiles = ((size_t)f.fcells + zl::SCAN_TILE - 1) / zl::SCAN_TILE;
+        const size_t sizes[9] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.fcells * 4, mb * cfg->n_workers * 4,
+                                 mb * (size_t)f.list1cap * 8, mb * f.nbk * 4, mb * f.nbk * f.capb * 8, mb * tiles * 4, 64};
+        void **ptrs[9] = {(void **)&f.table, (void **)&f.rowhint, (void **)&f.cellmax, (void **)&f.rcnt,
+                          (void **)&f.list1, (void **)&f.bcnt, (void **)&f.list2, (void **)&f.tilemax, (void **)&f.flags};
+        for (int i = 0; i < 9; ++i) {
             if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
             filter_b += sizes[i];
         }
@@ -1233,7 +1354,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         zl_status st = cuda_fail(nullptr, e);
         cudaFree(h->d_meta); cudaFree(h->d_seg);
         cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
-        cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2);
+        cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
         delete h;
         return st;
     }
@@ -1295,7 +1416,7 @@ zl_status zl_destroy(zl_handle *h) {
     cudaSetDevice(h->cfg.device);
     cudaFree(h->d_meta); cudaFree(h->d_seg);
     cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
-    cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2);
+    cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
     cudaFree(h->s_ts); cudaFree(h->s_idx); cudaFree(h->s_barrier); cudaFree(h->s_wait); cudaFree(h->s_status);
     if (h->s_stream) cudaStreamDestroy(h->s_stream);
     zl_profile_end(h);
@@ -1336,7 +1457,7 @@ size_t zl_workspace_bytes(const zl_handle *h) { return h ? h->ws_bytes + h->stag
 int32_t zl_launches_per_call(const zl_handle *h) {
     if (!h) return 0;
     const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter;
-    return 3 + (filter ? 5 : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
+    return 3 + (filter ? 6 : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
 }
 int32_t zl_segments_per_instance(const zl_handle *h, int32_t B) { return h && B >= 1 ? make_plan(h, B).nseg : 0; }
 int32_t zl_last_cuda_error(const zl_handle *h) { return h ? h->last_cuda_error : 0; }

@@ -195,7 +195,7 @@ def test_host_detected_errors():
         h.select_batched(ts)             # B > max_batch
     with pytest.raises(zl.ZipLineError):
         h.set_option("no_such_option", 1)
-    assert h.launches_per_call == 8 and h.workspace_bytes > 0
+    assert h.launches_per_call == 9 and h.workspace_bytes > 0
     h.destroy()
 
 
