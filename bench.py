@@ -262,8 +262,8 @@ def main():
     lmin = ts_np[:, :, -1].min(axis=1)
     examined = int((ts_np <= lmin[:, None, None]).sum()) if objective == 0 else nts
     def dominant(pr):
-        stages = {"k_prologue": pr["ms_prologue"], "k_filter": pr["ms_filter"], "k_small+k_sweep": pr["ms_sweep"],
-                  "k_finalize": pr["ms_finalize"]}
+        stages = {"k_prologue": pr["ms_prologue"], "k_filter": pr["ms_filter"],
+                  "k_tail+k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep": pr["ms_sweep"], "k_finalize": pr["ms_finalize"]}
         name = max(stages, key=stages.get)
         return name, stages[name] / pr["calls"]
 

@@ -118,6 +118,7 @@ constexpr int FILTER_MAX_CELLS = 8192;
 
 __global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int R, int objective, int flags,
                                                     InstMeta *meta, FilterBufs F) {
+    grid_dep_wait();
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
     const int64_t *inst = ts + (size_t)b * n * R;
     __shared__ uint64_t s[4][32];
@@ -331,6 +332,7 @@ __device__ __forceinline__ uint32_t filter_half(const FilterCtx &C, const int64_
 
 __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R, int flags, int rows_per_cta,
                                                   InstMeta *meta, FilterBufs F) {
+    grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ unsigned int scount;
     const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
@@ -437,6 +439,7 @@ constexpr int SCAN_TILE = 4096;
 
 // pass 1: maximum of every tile of SCAN_TILE fine cells.  A fixed grid walks the (tile, instance) pairs.
 __global__ void __launch_bounds__(256) k_tilemax(const InstMeta *meta, FilterBufs F, int B) {
+    grid_dep_wait();
     __shared__ uint64_t tmp[34];
     if (F.flags[0] == 0) return;                                  // no instance takes this route in this call
     const int tid = threadIdx.x, nt = blockDim.x;
@@ -459,6 +462,7 @@ __global__ void __launch_bounds__(256) k_tilemax(const InstMeta *meta, FilterBuf
 // cells, floored by t0: coalesced in, every thread scans a run of consecutive cells in shared memory,
 // coalesced out.
 __global__ void __launch_bounds__(256) k_cellscan(const InstMeta *meta, FilterBufs F, int B) {
+    grid_dep_wait();
     __shared__ uint64_t tmp[34];
     __shared__ uint32_t tile[SCAN_TILE];
     if (F.flags[0] == 0) return;
@@ -491,6 +495,7 @@ __global__ void __launch_bounds__(256) k_cellscan(const InstMeta *meta, FilterBu
 }
 
 __global__ void __launch_bounds__(256) k_refine(InstMeta *meta, FilterBufs F, int B) {
+    grid_dep_wait();
     if (F.flags[0] == 0) return;
     const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
     const int cpb_shift = __ffs(F.fcells / F.nbk) - 1;            // fine cells per bucket is a power of two
@@ -536,6 +541,7 @@ __global__ void __launch_bounds__(256) k_refine(InstMeta *meta, FilterBufs F, in
 
 // Optional full check that every row is non-decreasing.
 __global__ void k_check_sorted(const int64_t *ts, int n, int R, size_t total, InstMeta *meta) {
+    grid_dep_wait();
     const size_t per = (size_t)n * R;
     for (size_t f = (size_t)blockIdx.x * blockDim.x + threadIdx.x; f < total; f += (size_t)gridDim.x * blockDim.x) {
         if ((f % R) == 0) continue;
@@ -824,6 +830,7 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
 
 template <int OBJ>
 __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
+    grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ SweepShared sh;
     uint32_t *curA = (uint32_t *)smem;
@@ -857,6 +864,7 @@ __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
 // time order, packs whole buckets into shared-memory batches and runs each batch with the running
 // maximum of `next` over everything before it (the prefix maximum of cellmax up to the batch's first cell).
 __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg, int B) {
+    grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
     __shared__ unsigned int sstatus, fill;
@@ -928,6 +936,7 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
 // start), then sorts what is left and sweeps it.  Dropped survivors never hold the running maximum
 // alone, so nothing has to be carried in.
 __global__ void __launch_bounds__(1024) k_tail(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg) {
+    grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
     __shared__ unsigned int sstatus, fill;
@@ -993,6 +1002,7 @@ __global__ void __launch_bounds__(1024) k_tail(const InstMeta *meta, FilterBufs 
 __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int R, int nseg, FilterBufs F, int nres,
                                                   int objective, int filter, const InstMeta *meta, const SegResult *seg,
                                                   int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
+    grid_dep_wait();
     const int b = blockIdx.y, tid = threadIdx.x;
     const InstMeta M = meta[b];
     __shared__ uint64_t red[34];
@@ -1157,7 +1167,7 @@ struct zl_handle {
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off;
     int last_cuda_error;
     int launches;
     // optional per-kernel timing: PROF_EVENTS events per recorded call
@@ -1179,8 +1189,24 @@ struct Pipeline {
     zl::InstMeta *meta; zl::SegResult *seg; int nres;
     zl::FilterBufs fb;                                            // fb.table == nullptr: no filter route
     int filter_threads, filter_rows;                              // 0: automatic
+    int pdl_off;                                                  // bit mask of kernels launched without early scheduling
     int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;
 };
+
+// Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in
+// the stream is still running; every kernel here waits for that predecessor (grid_dep_wait) before it
+// touches memory.
+template <typename... KArgs, typename... Args>
+void launch_dep(bool early, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = early ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_t *ev) {
     const bool filter = q.fb.table != nullptr && q.objective == ZL_OBJ_RANGE;
@@ -1192,7 +1218,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     if (q.flags & ZL_FLAG_CHECK_SORTED) {
         const size_t total = (size_t)q.B * q.n * q.R;
         const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)q.num_sms * 16);
-        zl::k_check_sorted<<<blocks, 256, 0, st>>>(q.ts, q.n, q.R, total, q.meta);
+        launch_dep(!((q.pdl_off >> 0) & 1), zl::k_check_sorted, dim3(blocks), dim3(256), 0, st, q.ts, q.n, q.R, total, q.meta);
     }
     if (ev) cudaEventRecord(ev[1], st);
     if (filter) {
@@ -1205,19 +1231,21 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         fb.nreg = (int)((q.n + rpc - 1) / rpc);
         fb.regcap = fb.list1cap / fb.nreg;
         const size_t fsmem = (size_t)fb.cells * 4 + (size_t)nw * zl::FILTER_STAGES * zl::FILTER_SLOT * 8;
-        zl::k_filter<<<dim3(fb.nreg, q.B), threads, fsmem, st>>>(q.ts, q.n, q.R, q.flags, (int)rpc, q.meta, fb);
+        launch_dep(!((q.pdl_off >> 1) & 1), zl::k_filter, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.flags, (int)rpc, q.meta, fb);
         if (ev) cudaEventRecord(ev[2], st);
         const int tcap = (int)std::min<long long>((long long)zl::TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
-        zl::k_tail<<<q.B, std::max(64, std::min(1024, tcap / 2)), (size_t)tcap * 8 + (size_t)fb.cells * 4, st>>>(q.meta, fb, q.n, q.nres, q.seg);
+        launch_dep(!((q.pdl_off >> 2) & 1), zl::k_tail, dim3(q.B), dim3(std::max(64, std::min(1024, tcap / 2))), (size_t)tcap * 8 + (size_t)fb.cells * 4, st,
+                   (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg);
         // the route for instances with many survivors: fixed-size grids that return at once when no instance needs them
         const int tiles = (fb.fcells + zl::SCAN_TILE - 1) / zl::SCAN_TILE;
         const int wide = 4 * q.num_sms;
-        zl::k_tilemax<<<std::min(tiles * q.B, wide), 256, 0, st>>>(q.meta, fb, q.B);
-        zl::k_cellscan<<<std::min(tiles * q.B, wide), 256, 0, st>>>(q.meta, fb, q.B);
-        zl::k_refine<<<std::min(fb.nreg * q.B, wide), 256, 0, st>>>(q.meta, fb, q.B);
+        launch_dep(!((q.pdl_off >> 3) & 1), zl::k_tilemax, dim3(std::min(tiles * q.B, wide)), dim3(256), 0, st, (const zl::InstMeta *)q.meta, fb, q.B);
+        launch_dep(!((q.pdl_off >> 4) & 1), zl::k_cellscan, dim3(std::min(tiles * q.B, wide)), dim3(256), 0, st, (const zl::InstMeta *)q.meta, fb, q.B);
+        launch_dep(!((q.pdl_off >> 5) & 1), zl::k_refine, dim3(std::min(fb.nreg * q.B, wide)), dim3(256), 0, st, q.meta, fb, q.B);
         const int ngroups = (fb.nbk + fb.grp - 1) / fb.grp;
         const int bthreads = std::max(64, std::min(256, fb.capb / 4));
-        zl::k_buckets<<<std::min(ngroups * q.B, wide), bthreads, (size_t)fb.capb * 8, st>>>(q.meta, fb, q.n, q.nres, q.seg, q.B);
+        launch_dep(!((q.pdl_off >> 6) & 1), zl::k_buckets, dim3(std::min(ngroups * q.B, wide)), dim3(bthreads), (size_t)fb.capb * 8, st,
+                   (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg, q.B);
     } else if (ev) {
         cudaEventRecord(ev[2], st);
     }
@@ -1229,11 +1257,11 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     // with the filter route on, the segment sweep is only the fallback: a small persistent grid
     const int items = p.nseg * q.B;
     const int sweep_ctas = filter ? std::min(items, 2 * q.num_sms) : items;
-    if (q.objective == ZL_OBJ_RANGE) zl::k_sweep<ZL_OBJ_RANGE><<<sweep_ctas, p.threads, p.smem, st>>>(sp);
-    else zl::k_sweep<ZL_OBJ_SUM><<<sweep_ctas, p.threads, p.smem, st>>>(sp);
+    if (q.objective == ZL_OBJ_RANGE) launch_dep(!((q.pdl_off >> 7) & 1), zl::k_sweep<ZL_OBJ_RANGE>, dim3(sweep_ctas), dim3(p.threads), p.smem, st, sp);
+    else launch_dep(!((q.pdl_off >> 7) & 1), zl::k_sweep<ZL_OBJ_SUM>, dim3(sweep_ctas), dim3(p.threads), p.smem, st, sp);
     if (ev) cudaEventRecord(ev[3], st);
     const int fthreads = std::max(32, std::min(256, pow2_ceil(q.n)));
-    zl::k_finalize<<<dim3((q.n + fthreads - 1) / fthreads, q.B), fthreads, 0, st>>>(q.ts, q.n, q.R, p.nseg, fb, q.nres, q.objective,
+    launch_dep(!((q.pdl_off >> 8) & 1), zl::k_finalize, dim3((q.n + fthreads - 1) / fthreads, q.B), dim3(fthreads), 0, st, q.ts, q.n, q.R, p.nseg, fb, q.nres, q.objective,
                                                                   filter ? 1 : 0, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
     if (ev) cudaEventRecord(ev[4], st);
 }
@@ -1441,6 +1469,8 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
     } else if (!strcmp(key, "filter_threads")) {
         if (value && (!is_pow2(value) || value < 64 || value > 1024)) return ZL_ERR_INVALID_ARG;
         h->opt_filter_threads = value;
+    } else if (!strcmp(key, "pdl_off")) {
+        h->opt_pdl_off = value;                 // bit k set: kernel k of the chain is launched without early scheduling
     } else if (!strcmp(key, "filter_rows")) {
         if (value > 65536) return ZL_ERR_INVALID_ARG;
         h->opt_filter_rows = value;
@@ -1479,7 +1509,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.ts = d_ts; q.B = B; q.n = n; q.R = R; q.objective = obj; q.flags = h->cfg.flags; q.num_sms = h->num_sms;
     q.meta = h->d_meta; q.seg = h->d_seg; q.nres = h->nres;
     q.fb = h->fb;
-    q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows;
+    q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.pdl_off = h->opt_pdl_off;
     if (h->opt_no_filter) q.fb.table = nullptr;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, st, ev);
@@ -1620,7 +1650,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
     q.meta = meta; q.seg = seg; q.nres = p.nseg;
     memset(&q.fb, 0, sizeof(q.fb));
-    q.filter_threads = q.filter_rows = 0;
+    q.filter_threads = q.filter_rows = 0; q.pdl_off = 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr);
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;

@@ -131,6 +131,13 @@ __device__ __forceinline__ T warp_reduce(T x, Op op) {
     return x;
 }
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute has its
+// launch prepared while its predecessor in the stream is still running.  grid_dep_wait() blocks until
+// the predecessor grid has completed and its writes are visible (a no-op for a normally launched
+// kernel); every kernel of the chain calls it first.  No kernel signals early: dependents that became
+// resident while a long kernel was still running slowed that kernel down.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ int64_t ldg64(const int64_t *p) { return (int64_t)__ldg((const long long *)p); }
 
 }  // namespace zl
