@@ -25,7 +25,7 @@
 
 namespace zl {
 
-constexpr int MAX_WORKERS = 8192;
+constexpr int MAX_WORKERS = 4096;
 constexpr int MAX_SEGMENTS = 256;
 constexpr int TRACE_MAX = 4096;
 constexpr int64_t VALUE_LIMIT = (int64_t)1 << 62;
@@ -97,7 +97,7 @@ __device__ __forceinline__ uint32_t cell_of(uint32_t T, uint32_t cscale) { retur
 
 // Instances with at most this many survivors of the filter pass are finished by one CTA (k_tail);
 // larger ones go through cell scan, refinement and the bucket sweep.
-constexpr uint32_t TAIL_CAP = 8192;
+constexpr uint32_t TAIL_CAP = 2048;
 __device__ __forceinline__ bool tail_instance(const InstMeta &M) { return M.count <= TAIL_CAP; }
 
 // ------------------------------------------------------------------------------ prologue
@@ -116,7 +116,7 @@ __device__ __forceinline__ bool tail_instance(const InstMeta &M) { return M.coun
 constexpr int FILTER_ROWS = 32;      // rows that build the table
 constexpr int FILTER_MAX_CELLS = 8192;
 
-__global__ void __launch_bounds__(1024) k_prologue(const int64_t *ts, int n, int R, int objective, int flags,
+__global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, int R, int objective, int flags,
                                                     InstMeta *meta, FilterBufs F) {
     grid_dep_wait();
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
@@ -553,15 +553,27 @@ __global__ void k_check_sorted(const int64_t *ts, int n, int R, size_t total, In
 // Sort the batch into time order, scan it and evaluate every candidate; per-thread best is kept
 // in (bd, bt).  RANGE: carry = max of `next` over everything before the batch.  SUM: carryS/carryC =
 // sum of the latest element / number of started workers before the batch.
+// Shared-memory workspace of a batch: `in` receives the nodes, `out` their sorted order.
+template <typename K> struct BatchWS { Key<K> *in, *out; uint32_t *cnt; int cap; };
+
 template <typename K, int OBJ>
-__device__ void run_batch(Key<K> *keys, int m, K t0, int n, uint64_t *tmp64, K carryMax, uint64_t &carryS,
+__device__ void run_batch(const BatchWS<K> &ws, int m, K t0, int n, uint64_t *tmp64, K carryMax, uint64_t &carryS,
                           uint32_t &carryC, uint64_t &bd, uint64_t &bt) {
     if (m == 0) return;
-    int P = 64;
-    while (P < m) P <<= 1;
-    for (int i = m + threadIdx.x; i < P; i += blockDim.x) keys[i] = Key<K>::inf();
-    __syncthreads();
-    bitonic_sort(keys, P);
+    const Key<K> *keys;
+    if (m <= 256) {
+        // small batches: the comparison network (mostly warp-local steps) beats the bookkeeping of the slot sort
+        int P2 = 64;
+        while (P2 < m) P2 <<= 1;
+        for (int i = m + threadIdx.x; i < P2; i += blockDim.x) ws.in[i] = Key<K>::inf();
+        __syncthreads();
+        bitonic_sort(ws.in, P2);
+        keys = ws.in;
+    } else {
+        slot_sort<K>(ws.in, ws.out, ws.cnt, ws.cap, m, ws.cap, tmp64);
+        keys = ws.out;
+    }
+    const int P = m;
     const int ipt = (P + blockDim.x - 1) / blockDim.x;
     const int k0 = threadIdx.x * ipt, k1 = min(k0 + ipt, m);
     if (OBJ == ZL_OBJ_RANGE) {
@@ -646,7 +658,8 @@ struct SweepShared {
 
 template <typename K, int OBJ>
 __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int64_t *inst, SweepShared &sh,
-                              uint32_t *curA, uint32_t *curB, Key<K> *keys, int seg_index, SegResult &out) {
+                              uint32_t *curA, uint32_t *curB, const BatchWS<K> &ws, int seg_index, SegResult &out) {
+    Key<K> *keys = ws.in;
     const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
     const int n = P.n, R = P.R, G = P.G, NG = nt / G;
     const int gi = tid / G, g = tid % G;
@@ -794,7 +807,7 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
             if (overflow) {
                 // the round does not fit: flush what was there, or shorten the window; cursors are not committed
                 if (count_before > 0) {
-                    run_batch<K, OBJ>(keys, (int)count_before, t0, n, sh.tmp, carryMax, carryS, carryC, bd, bt);
+                    run_batch<K, OBJ>(ws, (int)count_before, t0, n, sh.tmp, carryMax, carryS, carryC, bd, bt);
                     carryMax = floorv;
                     count_before = 0;
                 } else {
@@ -814,7 +827,7 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
                 delta = (uint64_t)fmaxf(1.f, fminf((float)delta * f, 4.0e18f));
             }
             if (count_before > (uint32_t)(P.cap / 2)) {
-                run_batch<K, OBJ>(keys, (int)count_before, t0, n, sh.tmp, carryMax, carryS, carryC, bd, bt);
+                run_batch<K, OBJ>(ws, (int)count_before, t0, n, sh.tmp, carryMax, carryS, carryC, bd, bt);
                 carryMax = floorv;
                 count_before = 0;
                 if (tid == 0) sh.count = 0;
@@ -822,7 +835,7 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
             }
         }
         if (count_before > 0)
-            run_batch<K, OBJ>(keys, (int)count_before, t0, n, sh.tmp, carryMax, carryS, carryC, bd, bt);
+            run_batch<K, OBJ>(ws, (int)count_before, t0, n, sh.tmp, carryMax, carryS, carryC, bd, bt);
     }
 
     block_best_to_result(bd, bt, status, sh.tmp, &sh.status, out);
@@ -835,7 +848,10 @@ __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
     __shared__ SweepShared sh;
     uint32_t *curA = (uint32_t *)smem;
     uint32_t *curB = curA + P.n;
+    // shared memory: row cursors | batch nodes | sorted batch | slot counters
     unsigned char *kb = smem + (((size_t)2 * P.n * sizeof(uint32_t) + 15) & ~(size_t)15);
+    unsigned char *kb2 = kb + (size_t)P.cap * 8;
+    uint32_t *kcnt = (uint32_t *)(kb2 + (size_t)P.cap * 8);
     if (P.need && P.need[1] == 0) return;                        // the filter route finished every instance
     // a fixed number of CTAs walks the (instance, segment) pairs
     const int items = P.B * P.nseg;
@@ -850,11 +866,13 @@ __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
         }
         const int64_t *inst = P.ts + (size_t)b * P.n * P.R;
         if (M.use32) {
-            sweep_segment<uint32_t, OBJ>(P, M, inst, sh, curA, curB, (Key<uint32_t> *)kb, sidx, out);
+            const BatchWS<uint32_t> ws{(Key<uint32_t> *)kb, (Key<uint32_t> *)kb2, kcnt, P.cap};
+            sweep_segment<uint32_t, OBJ>(P, M, inst, sh, curA, curB, ws, sidx, out);
         } else {
             SweepParams Q = P;
             Q.cap = P.cap / 2;                      // 16-byte nodes: half as many fit
-            sweep_segment<uint64_t, OBJ>(Q, M, inst, sh, curA, curB, (Key<uint64_t> *)kb, sidx, out);
+            const BatchWS<uint64_t> ws{(Key<uint64_t> *)kb, (Key<uint64_t> *)kb2, kcnt, Q.cap};
+            sweep_segment<uint64_t, OBJ>(Q, M, inst, sh, curA, curB, ws, sidx, out);
         }
         __syncthreads();
     }
@@ -872,6 +890,7 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
     const int tid = threadIdx.x, nt = blockDim.x;
     const int ngroups = (F.nbk + F.grp - 1) / F.grp;
     Key<uint32_t> *keys = (Key<uint32_t> *)smem;
+    const BatchWS<uint32_t> ws{keys, keys + F.capb, (uint32_t *)(keys + 2 * (size_t)F.capb), F.capb};
     for (int item = blockIdx.x; item < ngroups * B; item += gridDim.x) {
     const int b = item / ngroups, g = item % ngroups;
     __syncthreads();                                              // shared state of the previous item is done with
@@ -907,7 +926,7 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
             for (uint32_t i = lane; i < c; i += 32) keys[off + i].w = src[i];
         }
         __syncthreads();
-        run_batch<uint32_t, ZL_OBJ_RANGE>(keys, (int)group_total, (uint32_t)M.t0, n, tmp, carry0, cs, cc, bd, bt);
+        run_batch<uint32_t, ZL_OBJ_RANGE>(ws, (int)group_total, (uint32_t)M.t0, n, tmp, carry0, cs, cc, bd, bt);
     } else {
         int m = 0;
         uint32_t carry_batch = carry0;
@@ -915,7 +934,7 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
             const int c = (int)min(bcnt[k], (uint32_t)F.capb);
             if (c == 0) continue;
             if (m + c > F.capb) {
-                run_batch<uint32_t, ZL_OBJ_RANGE>(keys, m, (uint32_t)M.t0, n, tmp, carry_batch, cs, cc, bd, bt);
+                run_batch<uint32_t, ZL_OBJ_RANGE>(ws, m, (uint32_t)M.t0, n, tmp, carry_batch, cs, cc, bd, bt);
                 carry_batch = g0[(size_t)k * cpb];        // G at the start of the next batch's first bucket
                 m = 0;
             }
@@ -924,7 +943,7 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
             m += c;
             __syncthreads();
         }
-        if (m > 0) run_batch<uint32_t, ZL_OBJ_RANGE>(keys, m, (uint32_t)M.t0, n, tmp, carry_batch, cs, cc, bd, bt);
+        if (m > 0) run_batch<uint32_t, ZL_OBJ_RANGE>(ws, m, (uint32_t)M.t0, n, tmp, carry_batch, cs, cc, bd, bt);
     }
     block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres + g]);
     }
@@ -935,7 +954,7 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
 // exclusive prefix maximum, drop every survivor whose next does not exceed the value at its cell's
 // start), then sorts what is left and sweeps it.  Dropped survivors never hold the running maximum
 // alone, so nothing has to be carried in.
-__global__ void __launch_bounds__(1024) k_tail(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg) {
+__global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg, int tcap) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
@@ -950,6 +969,7 @@ __global__ void __launch_bounds__(1024) k_tail(const InstMeta *meta, FilterBufs 
     if (M.status != ZL_OK || !handled_by_filter(M, 1) || !tail_instance(M)) return;
     uint32_t *g = (uint32_t *)smem;                               // [cells]
     Key<uint32_t> *keys = (Key<uint32_t> *)(smem + (size_t)F.cells * 4);
+    const BatchWS<uint32_t> ws{keys, keys + tcap, (uint32_t *)(keys + 2 * (size_t)tcap), tcap};
     const int cells = F.cells;
     for (int c = tid; c < cells; c += nt) g[c] = 0;
     if (tid == 0) { sstatus = 0; fill = 0; }
@@ -992,7 +1012,7 @@ __global__ void __launch_bounds__(1024) k_tail(const InstMeta *meta, FilterBufs 
     __syncthreads();
     uint64_t bd = ~0ull, bt = ~0ull, cs = 0;
     uint32_t cc = 0;
-    run_batch<uint32_t, ZL_OBJ_RANGE>(keys, (int)fill, (uint32_t)M.t0, n, tmp, (uint32_t)0, cs, cc, bd, bt);
+    run_batch<uint32_t, ZL_OBJ_RANGE>(ws, (int)fill, (uint32_t)M.t0, n, tmp, (uint32_t)0, cs, cc, bd, bt);
     block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres]);
 }
 
@@ -1167,7 +1187,7 @@ struct zl_handle {
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads;
     int last_cuda_error;
     int launches;
     // optional per-kernel timing: PROF_EVENTS events per recorded call
@@ -1190,6 +1210,7 @@ struct Pipeline {
     zl::FilterBufs fb;                                            // fb.table == nullptr: no filter route
     int filter_threads, filter_rows;                              // 0: automatic
     int pdl_off;                                                  // bit mask of kernels launched without early scheduling
+    int prologue_threads, tail_threads;                           // 0: automatic
     int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;
 };
 
@@ -1213,7 +1234,10 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     zl::FilterBufs fb = q.fb;
     if (!filter) memset(&fb, 0, sizeof(fb));
     if (ev) cudaEventRecord(ev[0], st);
-    const int pthreads = std::max(128, std::min(1024, pow2_ceil(q.n)));
+    // many small instances: small CTAs so that several share an SM; few large ones: one large CTA each
+    const bool many = q.B > 2 * q.num_sms;
+    const int pthreads = q.prologue_threads ? q.prologue_threads
+                         : many ? std::max(128, std::min(256, pow2_ceil(2 * q.n))) : std::max(512, std::min(1024, pow2_ceil(q.n)));
     zl::k_prologue<<<q.B, pthreads, 0, st>>>(q.ts, q.n, q.R, q.objective, q.flags, q.meta, fb);
     if (q.flags & ZL_FLAG_CHECK_SORTED) {
         const size_t total = (size_t)q.B * q.n * q.R;
@@ -1234,8 +1258,8 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         launch_dep(!((q.pdl_off >> 1) & 1), zl::k_filter, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.flags, (int)rpc, q.meta, fb);
         if (ev) cudaEventRecord(ev[2], st);
         const int tcap = (int)std::min<long long>((long long)zl::TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
-        launch_dep(!((q.pdl_off >> 2) & 1), zl::k_tail, dim3(q.B), dim3(std::max(64, std::min(1024, tcap / 2))), (size_t)tcap * 8 + (size_t)fb.cells * 4, st,
-                   (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg);
+        launch_dep(!((q.pdl_off >> 2) & 1), zl::k_tail, dim3(q.B), dim3(q.tail_threads ? q.tail_threads : many ? (tcap <= 1024 ? 128 : 256) : std::max(64, std::min(1024, tcap / 2))), (size_t)tcap * 20 + (size_t)fb.cells * 4, st,
+                   (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg, tcap);
         // the route for instances with many survivors: fixed-size grids that return at once when no instance needs them
         const int tiles = (fb.fcells + zl::SCAN_TILE - 1) / zl::SCAN_TILE;
         const int wide = 4 * q.num_sms;
@@ -1244,7 +1268,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         launch_dep(!((q.pdl_off >> 5) & 1), zl::k_refine, dim3(std::min(fb.nreg * q.B, wide)), dim3(256), 0, st, q.meta, fb, q.B);
         const int ngroups = (fb.nbk + fb.grp - 1) / fb.grp;
         const int bthreads = std::max(64, std::min(256, fb.capb / 4));
-        launch_dep(!((q.pdl_off >> 6) & 1), zl::k_buckets, dim3(std::min(ngroups * q.B, wide)), dim3(bthreads), (size_t)fb.capb * 8, st,
+        launch_dep(!((q.pdl_off >> 6) & 1), zl::k_buckets, dim3(std::min(ngroups * q.B, wide)), dim3(bthreads), (size_t)fb.capb * 20, st,
                    (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg, q.B);
     } else if (ev) {
         cudaEventRecord(ev[2], st);
@@ -1284,7 +1308,7 @@ LaunchPlan make_plan(const zl_handle *h, int B) {
     if (p.G > p.threads) p.G = p.threads;
     // batch capacity in 8-byte nodes; wide (16-byte) instances get half, which must still hold one
     // node per worker
-    int cap = std::max(8192, pow2_ceil(2 * n));
+    int cap = std::max(4096, pow2_ceil(2 * n));
     const int small = std::max(pow2_ceil((int)std::min<long long>(N, 1 << 20)), std::max(pow2_ceil(2 * n), 128));
     p.cap = std::min(cap, small);
     // time segments per instance: enough CTAs to fill the GPU a few times over, each long enough to
@@ -1299,10 +1323,10 @@ LaunchPlan make_plan(const zl_handle *h, int B) {
     p.nseg = nseg;
     const int rf = h->opt_round_factor ? h->opt_round_factor : 75;
     long long target = (long long)n * std::max(p.G, 4) * rf / 100;
-    if (h->cfg.objective == ZL_OBJ_SUM) target = std::min<long long>(target, (long long)p.cap * 45 / 100 / 2);
+    if (h->cfg.objective == ZL_OBJ_SUM) target = std::min<long long>(target, (long long)p.cap * 45 / 100);
     target = std::min<long long>(target, (long long)p.cap * 4);
     p.target = (int)std::max<long long>(target, 32);
-    p.smem = (((size_t)2 * n * sizeof(uint32_t) + 15) & ~(size_t)15) + (size_t)p.cap * 8;
+    p.smem = (((size_t)2 * n * sizeof(uint32_t) + 15) & ~(size_t)15) + (size_t)p.cap * 20;   // nodes, sorted nodes, slot counters
     return p;
 }
 
@@ -1469,6 +1493,9 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
     } else if (!strcmp(key, "filter_threads")) {
         if (value && (!is_pow2(value) || value < 64 || value > 1024)) return ZL_ERR_INVALID_ARG;
         h->opt_filter_threads = value;
+    } else if (!strcmp(key, "prologue_threads") || !strcmp(key, "tail_threads")) {
+        if (value && (!is_pow2(value) || value < 64 || value > 1024)) return ZL_ERR_INVALID_ARG;
+        (key[0] == 'p' ? h->opt_prologue_threads : h->opt_tail_threads) = value;
     } else if (!strcmp(key, "pdl_off")) {
         h->opt_pdl_off = value;                 // bit k set: kernel k of the chain is launched without early scheduling
     } else if (!strcmp(key, "filter_rows")) {
@@ -1510,6 +1537,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.meta = h->d_meta; q.seg = h->d_seg; q.nres = h->nres;
     q.fb = h->fb;
     q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.pdl_off = h->opt_pdl_off;
+    q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
     if (h->opt_no_filter) q.fb.table = nullptr;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, st, ev);
@@ -1650,7 +1678,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
     q.meta = meta; q.seg = seg; q.nres = p.nseg;
     memset(&q.fb, 0, sizeof(q.fb));
-    q.filter_threads = q.filter_rows = 0; q.pdl_off = 0;
+    q.filter_threads = q.filter_rows = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr);
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;

@@ -124,6 +124,76 @@ __device__ T block_scan_excl(T x, Op op, T identity, T *tmp, T *total) {
     return exc;
 }
 
+// ---------------------------------------------------------------------------------- slot sort
+// Sort in[0..m) by (time, payload) into out[0..m): a counting sort on the time (nslots time slots
+// between the batch's earliest and latest time, about one key per slot), then an insertion sort of
+// the few keys that share a slot.  A batch in which one slot holds more than SLOT_MAX keys falls back
+// to the bitonic network.  cnt: nslots words of shared memory; in and out hold cap >= m keys
+// (cap a power of two >= 64); tmp: 34 shared 64-bit words.  All threads of the block call it.
+constexpr int SLOT_MAX = 24;
+
+template <typename K>
+__device__ void slot_sort(Key<K> *in, Key<K> *out, uint32_t *cnt, int nslots, int m, int cap, uint64_t *tmp) {
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+    // range of times in the batch
+    K lo = ~(K)0, hi = 0;
+    for (int i = tid; i < m; i += nt) { const K t = in[i].t(); lo = min(lo, t); hi = max(hi, t); }
+    lo = warp_reduce(lo, OpMin()); hi = warp_reduce(hi, OpMax());
+    K *red = (K *)tmp;                                            // 32 entries of at most 8 bytes
+    if (lane == 0) red[warp] = lo;
+    for (int s = tid; s < nslots; s += nt) cnt[s] = 0;
+    __syncthreads();
+    for (int w = 0; w < nw; ++w) lo = min(lo, red[w]);
+    __syncthreads();
+    if (lane == 0) red[warp] = hi;
+    __syncthreads();
+    for (int w = 0; w < nw; ++w) hi = max(hi, red[w]);
+    __syncthreads();
+    int sh = 0;
+    while (((hi - lo) >> sh) >= (K)nslots) ++sh;                  // slot = (t - lo) >> sh < nslots, monotone in t
+    for (int i = tid; i < m; i += nt) atomicAdd(&cnt[(uint32_t)((in[i].t() - lo) >> sh)], 1u);
+    __syncthreads();
+    {   // exclusive prefix sum of the slot counts, in place; a slot that is too full is noted on the way
+        const int per = (nslots + nt - 1) / nt;
+        const int s0 = min(tid * per, nslots), s1 = min(s0 + per, nslots);
+        uint32_t loc = 0, big = 0;
+        for (int s = s0; s < s1; ++s) { loc += cnt[s]; big |= cnt[s] > (uint32_t)SLOT_MAX; }
+        uint32_t tot;
+        uint32_t run = block_scan_excl<uint32_t>(loc, OpAdd(), 0u, (uint32_t *)tmp, &tot);
+        for (int s = s0; s < s1; ++s) { const uint32_t c = cnt[s]; cnt[s] = run; run += c; }
+        uint32_t anybig;
+        block_scan_excl<uint32_t>(big, OpMax(), 0u, (uint32_t *)tmp, &anybig);
+        if (anybig) {
+            // many equal or nearly equal times: the comparison network handles any distribution
+            int P = 64;
+            while (P < m) P <<= 1;
+            for (int i = m + tid; i < P; i += nt) in[i] = Key<K>::inf();
+            __syncthreads();
+            bitonic_sort(in, P);
+            for (int i = tid; i < m; i += nt) out[i] = in[i];
+            __syncthreads();
+            return;
+        }
+    }
+    __syncthreads();
+    for (int i = tid; i < m; i += nt) {
+        const Key<K> k = in[i];
+        out[atomicAdd(&cnt[(uint32_t)((k.t() - lo) >> sh)], 1u)] = k;      // cnt[s] ends as the end of slot s
+    }
+    __syncthreads();
+    for (int s = tid; s < nslots; s += nt) {
+        const int e = (int)cnt[s], b = s ? (int)cnt[s - 1] : 0;
+        for (int i = b + 1; i < e; ++i) {                        // insertion sort of the slot's keys
+            const Key<K> k = out[i];
+            int j = i - 1;
+            while (j >= b && out[j] > k) { out[j + 1] = out[j]; --j; }
+            out[j + 1] = k;
+        }
+    }
+    __syncthreads();
+    (void)cap;
+}
+
 template <typename T, typename Op>
 __device__ __forceinline__ T warp_reduce(T x, Op op) {
 #pragma unroll
