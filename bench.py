@@ -36,6 +36,21 @@ CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.ac
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
 
+def recorded_traffic(key):
+    """DRAM bytes per launch from the committed ncu capture, or None once the kernel sources have changed since."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
+            rec = json.load(f)
+        hsh = hashlib.sha256()
+        for name in ("zipline.cu", "zl_device.cuh"):
+            with open(os.path.join(ROOT, "paper_2001_01347_b200", "csrc", name), "rb") as f:
+                hsh.update(f.read())
+        return rec.get(key) if rec.get("source_sha256") == hsh.hexdigest() else None
+    except Exception:
+        return None
+
+
 def measured_peak_gbs():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -55,7 +70,7 @@ class ClockSampler:
         try:
             self.f = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.idx}", f"--query-gpu={CLOCK_QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=self.f, stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -148,7 +163,7 @@ def workload_config(w, objective, gpus):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="zipline", choices=["zipline", "reference"])
     ap.add_argument("--workload", default="c4")
@@ -195,7 +210,7 @@ def main():
             h.set_option(k, int(v))
         return h
 
-    def timed(h, steps, warmup, host=False):
+    def timed(h, steps, warmup, host=False, profile=False):
         sel = None
 
         def step(i):
@@ -209,7 +224,7 @@ def main():
             dist.barrier()
             torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        if not host:
+        if profile:
             h.profile_begin(steps)
         t0 = time.perf_counter()
         e0.record()
@@ -220,7 +235,7 @@ def main():
         wall_ms = (time.perf_counter() - t0) * 1e3
         ms = wall_ms if host else e0.elapsed_time(e1)          # the host path runs on the library's own stream
         prof = None
-        if not host:
+        if profile:
             prof = h.profile_read()
             h.profile_end()
         if world > 1:
@@ -233,8 +248,9 @@ def main():
     sampler = ClockSampler(local)
     h = make_handle(0)
     sampler.start()
-    ms, prof, sel = timed(h, args.steps, args.warmup)
-    clocks = sampler.stop()
+    ms, _, sel = timed(h, args.steps, args.warmup)                       # the headline: no per-stage events in the stream
+    psteps = max(3, min(args.steps, 50))
+    _, prof, _ = timed(h, psteps, 3, profile=True)                       # per-stage CUDA events (they serialise the stages)
     status_ok = bool((sel.status == 0).all().item())
     launches = h.launches_per_call * args.steps
     ms_step = ms / args.steps
@@ -242,9 +258,11 @@ def main():
 
     # the same search when every timestamp is examined (no early stop)
     hf = make_handle(zl.ZL_FLAG_FULL_SWEEP)
-    ms_f, prof_f, _ = timed(hf, max(3, args.steps // 2), 3)
     steps_f = max(3, args.steps // 2)
+    ms_f, _, _ = timed(hf, steps_f, 3)
+    _, prof_f, _ = timed(hf, psteps, 3, profile=True)
     hf.destroy()
+    clocks = sampler.stop()
 
     # end to end: host buffers in, host results out, through the C ABI
     e2e_steps = max(3, min(args.steps, 10))
@@ -272,13 +290,15 @@ def main():
     dom_f, sweep_ms_f = dominant(prof_f)
     ach_f = nts * 8 / (sweep_ms_f * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                "peak_kind": f"{peak_kind} copy bandwidth", "traffic": None,
+                "peak_kind": f"{peak_kind} copy bandwidth",
+                "traffic": recorded_traffic(f"{w.name}_{args.objective}_default_{dom}"),
                 "bytes_per_launch": examined * 8, "ms_per_launch": sweep_ms,
                 "bytes_model": "8 B per timestamp not after the first exhausted row (the search stops there)"
                 if objective == 0 else "8 B per timestamp"}
     full = {"value": nts / (ms_f / steps_f * 1e-3), "unit": "timestamps/s", "ms_per_step": ms_f / steps_f,
             "roofline": {"bound": "hbm", "kernel": dom_f, "achieved": ach_f, "peak": peak, "unit": "GB/s",
-                         "frac": ach_f / peak, "bytes_per_launch": nts * 8, "ms_per_launch": sweep_ms_f, "traffic": None}}
+                         "frac": ach_f / peak, "bytes_per_launch": nts * 8, "ms_per_launch": sweep_ms_f,
+                         "traffic": recorded_traffic(f"{w.name}_{args.objective}_full_{dom_f}")}}
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:
