@@ -40,13 +40,17 @@ def recorded_traffic(key):
     """DRAM bytes per launch from the committed ncu capture, or None once the kernel sources have changed since."""
     import hashlib
     try:
-        with open(os.path.join(ROOT, "profiles", "traffic.json")) as f:
-            rec = json.load(f)
+        rec = {}
+        with open(os.path.join(ROOT, "profiles", "k_filter_c4_traffic.txt")) as f:
+            for line in f:
+                if line.strip() and not line.startswith("#"):
+                    k, v = line.split()
+                    rec[k] = v
         hsh = hashlib.sha256()
         for name in ("zipline.cu", "zl_device.cuh"):
             with open(os.path.join(ROOT, "paper_2001_01347_b200", "csrc", name), "rb") as f:
                 hsh.update(f.read())
-        return rec.get(key) if rec.get("source_sha256") == hsh.hexdigest() else None
+        return int(rec[key]) if rec.get("source_sha256") == hsh.hexdigest() and key in rec else None
     except Exception:
         return None
 
