@@ -147,11 +147,13 @@ zl_status zl_profile_end(zl_handle *h);
  * claimed all device memory for its own pool, a service with a fixed memory budget
  * that forbids allocation after start-up, or a latency-critical loop that must not
  * take the driver's allocation lock (cudaMalloc and cudaFree can stall every stream
- * of the device).  zl_create allocates the search's scratch (per-instance summaries
- * and per-segment partial results) with cudaMalloc; this entry point keeps that
- * scratch in a fixed array compiled into the library instead, zl_noalloc_scratch_bytes()
+ * of the device).  zl_create allocates the search's scratch with cudaMalloc; this entry
+ * point keeps the scratch it needs (per-instance summaries and per-segment partial
+ * results) in a fixed array compiled into the library instead, zl_noalloc_scratch_bytes()
  * bytes (about 400 KB) that every GPU using the library holds until the process exits.
- * It calls no cudaMalloc, cudaFree or other allocating routine.
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  It always runs the
+ * segment sweep; the faster filter route of the RANGE objective needs buffers of about
+ * the size of the input and is only available through a handle.
  *
  * Arguments are those of zl_create's configuration (n_workers, lookahead_R, objective,
  * flags) followed by those of zl_select_batched, with the same meaning, layout and
