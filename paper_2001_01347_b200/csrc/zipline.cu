@@ -1308,7 +1308,7 @@ LaunchPlan make_plan(const zl_handle *h, int B) {
     if (p.G > p.threads) p.G = p.threads;
     // batch capacity in 8-byte nodes; wide (16-byte) instances get half, which must still hold one
     // node per worker
-    int cap = std::max(4096, pow2_ceil(2 * n));
+    int cap = std::max(h->cfg.objective == ZL_OBJ_SUM ? 8192 : 4096, pow2_ceil(2 * n));
     const int small = std::max(pow2_ceil((int)std::min<long long>(N, 1 << 20)), std::max(pow2_ceil(2 * n), 128));
     p.cap = std::min(cap, small);
     // time segments per instance: enough CTAs to fill the GPU a few times over, each long enough to
