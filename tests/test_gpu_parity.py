@@ -229,3 +229,46 @@ def test_trace_matches_oracle_trace():
             ref = o.trace(ts[b])
             for k in ref:
                 assert (tr[k][b].cpu().numpy() == ref[k]).all(), (k, n, R, b)
+
+
+# ---------------------------------------------------------------- the three RANGE routes
+def _routes(ts_np):
+    B, n, R = ts_np.shape
+    h = zl.ZipLine(n, R, B, 0)
+    sel = h.select_batched(torch.from_numpy(ts_np).cuda())
+    torch.cuda.synchronize()
+    filtered, refined, overflow = h.filter_counts(B)
+    h.destroy()
+    return sel, np.array(filtered), np.array(refined), np.array(overflow)
+
+
+def test_range_routes_are_all_exercised_and_exact():
+    # few survivors: finished by the single-CTA tail
+    ts = zi.generate(zi.CONFIGS["c4"].with_(B=3, n=256, R=512))
+    sel, filtered, refined, overflow = _routes(ts)
+    assert (overflow == 0).all() and (filtered <= 2048).all() and (filtered > 0).all()
+    assert_same(ts, 0, (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()))
+    # one common period per half of the workers: many elements raise the running maximum, so the
+    # instance goes through cell scan, refinement and the bucket sweep
+    ts = zi.generate(zi.CONFIGS["c5"].with_(B=3, n=512, R=1024))
+    sel, filtered, refined, overflow = _routes(ts)
+    assert (overflow == 0).all() and (filtered > 2048).all() and (refined > 0).all() and (refined <= filtered).all()
+    assert_same(ts, 0, (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()))
+    # identical rows: every element survives, the lists overflow, the segment sweep takes over
+    row = np.cumsum(np.arange(1, 401))
+    ts = np.broadcast_to(row, (2, 200, 400)).astype(np.int64).copy()
+    sel, filtered, refined, overflow = _routes(ts)
+    assert (overflow == 1).all()
+    assert_same(ts, 0, (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()))
+
+
+def test_mixed_batch_of_routes():
+    # one batch holding a light, a heavy and an overflowing instance: the per-call flags must not let one starve another
+    n, R = 256, 512
+    light = zi.generate(zi.CONFIGS["c4"].with_(B=1, n=n, R=R))[0]
+    heavy = zi.generate(zi.CONFIGS["c5"].with_(B=1, n=n, R=R))[0]
+    same = np.broadcast_to(np.cumsum(np.arange(1, R + 1)) * 1000, (n, R)).astype(np.int64)
+    ts = np.stack([light, heavy, same, light + 7, heavy + 11])
+    sel, filtered, refined, overflow = _routes(ts)
+    assert overflow.tolist() == [0, 0, 1, 0, 0]
+    assert_same(ts, 0, (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()))
