@@ -64,7 +64,7 @@ struct FilterBufs {
     uint32_t *tilemax;   // [B][fcells/4096]  max of cellmax per tile of 4096 fine cells (scratch of the cell scan)
     uint32_t *rcnt;      // [B][nreg]         survivors per region (one region per CTA of the filter pass)
     uint64_t *list1;     // [B][list1cap]     survivors of the filter pass as (T << 32 | next), by region
-    uint32_t *flags;     // [2]               per call: [0] some instance needs scan/refine/buckets, [1] some needs the segment sweep
+    uint32_t *flags;     // [3]               per call: some instance needs [0] scan/refine/buckets, [1] the segment sweep, [2] k_finalize
     uint32_t *bcnt;      // [B][nbk]          survivors of the refinement per bucket
     uint64_t *list2;     // [B][nbk][capb]    survivors of the refinement
     int32_t cells, fcells, nbk, capb, grp;   // grp: fewest buckets per CTA of the bucket sweep
@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, 
     }
     __syncthreads();
     const InstMeta M = sm;
-    if (b == 0 && tid < 2 && F.flags) F.flags[tid] = 0;
+    if (b == 0 && tid < 3 && F.flags) F.flags[tid] = 0;
     if (M.cscale != 0) {
         const uint32_t cells = (uint32_t)F.cells, cscale = M.cscale, lmin = (uint32_t)M.lmin;
         const uint32_t wcell = 0xffffffffu / cscale + 2;          // > 2^32 / cscale
@@ -949,22 +949,55 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
     }
 }
 
+// Index of the last element of a sorted row that is <= bar (-1 if none).  Rows are close to arithmetic, so the
+// position is first guessed from the row's end points, bracketed by doubling steps around the guess, then bisected.
+__device__ int last_index_not_after(const int64_t *row, int R, int64_t bar) {
+    const int64_t e0 = ldg64(row), eR = ldg64(row + R - 1);
+    if (bar < e0) return -1;
+    if (bar >= eR) return R - 1;
+    // e0 <= bar < eR, R >= 2.  Invariant: row[lo - 1] <= bar, row[hi] > bar
+    int lo, hi;
+    int g = (int)((double)(bar - e0) * (double)(R - 1) / (double)(eR - e0));
+    g = max(0, min(g, R - 2));
+    if (ldg64(row + g) <= bar) {
+        lo = g + 1; hi = R - 1;
+        for (int step = 1; lo < hi; step <<= 1) {
+            const int q = min(lo + step - 1, hi - 1);
+            if (ldg64(row + q) <= bar) lo = q + 1; else { hi = q; break; }
+        }
+    } else {
+        hi = g; lo = 1;
+        for (int step = 1; lo < hi; step <<= 1) {
+            const int q = max(hi - step, lo);
+            if (ldg64(row + q) > bar) hi = q; else { lo = q + 1; break; }
+        }
+    }
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (ldg64(row + mid) <= bar) lo = mid + 1; else hi = mid;
+    }
+    return lo - 1;
+}
+
 // Instances with few survivors of the filter pass are finished by one CTA.  It first applies the
 // refinement at the resolution of the coarse cells, in shared memory (maximum of next per cell,
 // exclusive prefix maximum, drop every survivor whose next does not exceed the value at its cell's
 // start), then sorts what is left and sweeps it.  Dropped survivors never hold the running maximum
 // alone, so nothing has to be carried in.
-__global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg, int tcap) {
+__global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg, int tcap,
+                                                  const int64_t *ts, int R, int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
     __shared__ unsigned int sstatus, fill;
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
     const InstMeta M = meta[b];
-    if (M.status == ZL_OK && tid == 0) {
+    if (tid == 0) {
         // tell the later kernels of this call whether they have anything to do
-        if (!handled_by_filter(M, 1)) F.flags[1] = 1;
-        else if (!tail_instance(M)) F.flags[0] = 1;
+        const bool mine = M.status == ZL_OK && handled_by_filter(M, 1) && tail_instance(M);
+        if (M.status == ZL_OK && !handled_by_filter(M, 1)) F.flags[1] = 1;
+        else if (M.status == ZL_OK && !tail_instance(M)) F.flags[0] = 1;
+        if (!mine) F.flags[2] = 1;                                 // k_finalize has to write this instance's outputs
     }
     if (M.status != ZL_OK || !handled_by_filter(M, 1) || !tail_instance(M)) return;
     uint32_t *g = (uint32_t *)smem;                               // [cells]
@@ -1013,7 +1046,20 @@ __global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBu
     uint64_t bd = ~0ull, bt = ~0ull, cs = 0;
     uint32_t cc = 0;
     run_batch<uint32_t, ZL_OBJ_RANGE>(ws, (int)fill, (uint32_t)M.t0, n, tmp, (uint32_t)0, cs, cc, bd, bt);
-    block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres]);
+    __shared__ SegResult best;
+    block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, best);
+    __syncthreads();
+    // K5 for this instance right here: barrier, wait and the per-worker indices (k_finalize skips it)
+    const int fst = best.valid ? ZL_OK : ZL_ERR_TIMEOUT;          // a valid instance always has a candidate
+    const int64_t bar = fst == ZL_OK ? M.tmin + (int64_t)(best.t - 1) + (int64_t)best.d : INT64_MIN;
+    if (tid == 0) {
+        seg[(size_t)b * nres] = best;
+        wait[b] = fst == ZL_OK ? (int64_t)best.d : INT64_MIN;
+        barrier[b] = bar;
+        if (status) status[b] = fst;
+    }
+    for (int p = tid; p < n; p += nt)
+        idx[(size_t)b * n + p] = fst == ZL_OK ? last_index_not_after(ts + ((size_t)b * n + p) * R, R, bar) : -1;
 }
 
 // ------------------------------------------------------------------------------ finalize
@@ -1024,7 +1070,9 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
                                                   int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
     grid_dep_wait();
     const int b = blockIdx.y, tid = threadIdx.x;
+    if (filter && F.flags[2] == 0) return;                        // k_tail finished every instance of this call
     const InstMeta M = meta[b];
+    if (M.status == ZL_OK && handled_by_filter(M, filter) && tail_instance(M)) return;   // finished by k_tail
     __shared__ uint64_t red[34];
     __shared__ unsigned int sstatus;
     __shared__ SegResult best;
@@ -1061,34 +1109,7 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
     if (p < n) {
         int res = -1;
         if (fst == ZL_OK) {
-            const int64_t *row = ts + ((size_t)b * n + p) * R;
-            const int64_t e0 = ldg64(row), eR = ldg64(row + R - 1);
-            int lo, hi;                           // invariant: row[lo - 1] <= bar (or lo == 0), row[hi] > bar (or hi == R)
-            if (bar < e0) { lo = 0; hi = 0; }
-            else if (bar >= eR) { lo = R; hi = R; }
-            else {
-                // e0 <= bar < eR, R >= 2
-                int g = (int)((double)(bar - e0) * (double)(R - 1) / (double)(eR - e0));
-                g = max(0, min(g, R - 2));
-                if (ldg64(row + g) <= bar) {
-                    lo = g + 1; hi = R - 1;       // row[R-1] > bar
-                    for (int step = 1; lo < hi; step <<= 1) {
-                        const int q = min(lo + step - 1, hi - 1);
-                        if (ldg64(row + q) <= bar) lo = q + 1; else { hi = q; break; }
-                    }
-                } else {
-                    hi = g; lo = 1;               // row[0] <= bar
-                    for (int step = 1; lo < hi; step <<= 1) {
-                        const int q = max(hi - step, lo);
-                        if (ldg64(row + q) > bar) hi = q; else { lo = q + 1; break; }
-                    }
-                }
-                while (lo < hi) {
-                    const int mid = (lo + hi) >> 1;
-                    if (ldg64(row + mid) <= bar) lo = mid + 1; else hi = mid;
-                }
-            }
-            res = lo - 1;
+            res = last_index_not_after(ts + ((size_t)b * n + p) * R, R, bar);
         }
         idx[(size_t)b * n + p] = res;
     }
@@ -1259,7 +1280,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         if (ev) cudaEventRecord(ev[2], st);
         const int tcap = (int)std::min<long long>((long long)zl::TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
         launch_dep(!((q.pdl_off >> 2) & 1), zl::k_tail, dim3(q.B), dim3(q.tail_threads ? q.tail_threads : many ? (tcap <= 1024 ? 128 : 256) : std::max(64, std::min(1024, tcap / 2))), (size_t)tcap * 20 + (size_t)fb.cells * 4, st,
-                   (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg, tcap);
+                   (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg, tcap, q.ts, q.R, q.idx, q.barrier, q.wait, q.status);
         // the route for instances with many survivors: fixed-size grids that return at once when no instance needs them
         const int tiles = (fb.fcells + zl::SCAN_TILE - 1) / zl::SCAN_TILE;
         const int wide = 4 * q.num_sms;
