@@ -49,6 +49,8 @@ def _load():
         lib.zlo_alg2.restype = ci
         lib.zlo_trace.argtypes = [vp, ci, ci] + [vp] * 11
         lib.zlo_trace.restype = ci
+        lib.zlo_predict.argtypes = [vp, vp, ci, ci, vp]
+        lib.zlo_predict.restype = ci
         _lib = lib
     return _lib
 
@@ -113,6 +115,17 @@ def trace(M) -> dict:
     n, R = M.shape
     out = {k: np.empty(n * R, dtype=dt) for k, dt in TRACE_FIELDS}
     _check(_load().zlo_trace(M.ctypes.data, n, R, *[out[k].ctypes.data for k, _ in TRACE_FIELDS]))
+    return out
+
+
+def predict(last, interval, R: int) -> np.ndarray:
+    """Phase 1 of ZipLine: [n, R] future end timestamps, e_i = last + i * interval (i = 1..R)."""
+    last = np.ascontiguousarray(last, dtype=np.int64)
+    interval = np.ascontiguousarray(interval, dtype=np.int64)
+    if last.ndim != 1 or last.shape != interval.shape or R < 1:
+        raise ValueError("expected last[n], interval[n], R >= 1")
+    out = np.empty((last.shape[0], R), dtype=np.int64)
+    _check(_load().zlo_predict(last.ctypes.data, interval.ctypes.data, last.shape[0], int(R), out.ctypes.data))
     return out
 
 

@@ -33,6 +33,7 @@
  *                     the O(n) evaluation is too slow
  *   zlo_alg2          Algorithm 2 step by step (drop min(Z), refill until |Z|=n)
  *   zlo_trace         per-position intermediates of the pass, for kernel tests
+ *   zlo_predict       phase 1 of ZipLine: R future end timestamps per worker from its most recent interval
  *
  * Return codes: 0 ok, -1 bad argument, -2 a row is not non-decreasing,
  * -3 the objective does not fit int64, -4 out of memory.
@@ -312,5 +313,26 @@ int zlo_trace(const int64_t *M, int n, int R,
         if (nx > pm) pm = nx;
     }
     free(om);
+    return 0;
+}
+
+/* ---------------------------------------------------------------------- predictor
+ * Phase 1 of ZipLine (Introduction; Section II, first property; Section III): the future iteration
+ * intervals of a worker are predicted from its most recent interval under the stable-environment
+ * assumption.  The paper gives no formula; the reading taken is constant-interval extrapolation:
+ *   e^p_i = last[p] + i * interval[p],  i = 1..R
+ * last[p] = the worker's latest observed end timestamp, interval[p] >= 0 its most recent interval.
+ * out is [n][R].  Returns -1 on bad arguments, -3 if a value would reach 2^62. */
+int zlo_predict(const int64_t *last, const int64_t *interval, int n, int R, int64_t *out) {
+    if (!last || !interval || !out || n < 1 || R < 1) return -1;
+    const i128 limit = (i128)1 << 62;
+    for (int p = 0; p < n; ++p) {
+        if (last[p] < 0 || interval[p] < 0) return -1;
+        for (int i = 1; i <= R; ++i) {
+            i128 v = (i128)last[p] + (i128)i * interval[p];
+            if (v >= limit) return -3;
+            out[(size_t)p * R + (i - 1)] = (int64_t)v;
+        }
+    }
     return 0;
 }

@@ -1,16 +1,32 @@
 // ZipLine barrier-selection search for sm_100a: kernels and the C ABI (see include/zipline.h).
 //
-// One call runs, per instance of n sorted rows of R int64 timestamps:
-//   prologue   column scans: tmin, t0 = max_p e^p_1, lmin = min_p e^p_R, span
-//   sweep      the timeline is cut into time segments, one CTA each.  A CTA walks its segment in
-//              rounds: every row advances a cursor over the elements that fall in the round's time
-//              window (the rows are already sorted, so the n-way merge is a set of cursors), attaches
-//              to each element the payload the scan needs (next / delta+first flag), and appends it to
-//              a shared-memory batch.  A full batch is sorted into time order (Omega), scanned
-//              (prefix max of next / prefix sums of delta and flag) and evaluated, keeping the first
-//              minimum.  Carry-ins at a segment start come from per-row binary searches, so segments
-//              are independent.
-//   finalize   minimum over the segments of an instance, barrier, per-worker index recovery.
+// Per instance: n sorted rows of R int64 timestamps.  Every kernel of a call is enqueued on the caller's
+// stream with programmatic stream serialization and starts with grid_dep_wait().
+//
+//   k_prologue  column scans (tmin, t0 = max_p e^p_1, lmin = min_p e^p_R, span); for the RANGE filter
+//               route also the per-row estimates, the filter table and the per-call counters.
+//
+// RANGE (max(Z) - min(Z)), filter route: an element matters only if its `next` exceeds G, the running
+// maximum of `next` over everything earlier (floored by t0); see the comment above k_prologue.
+//   k_filter    one warp per row streams the row in storage order (cp.async ring), forms (T, next),
+//               tests it against the table and appends the survivors to per-CTA lists.
+//   k_tail      instances with few survivors: refine, sort into time order, prefix max of next,
+//               evaluate d = max(T, t0, PM) - T, keep the first minimum, recover the indices.
+//   k_tilemax, k_cellscan, k_refine, k_buckets
+//               instances with many survivors: G at every fine time cell, drop what cannot matter,
+//               bucket by time, sort + scan + evaluate per group of buckets.
+//
+// SUM (sum_p (max(Z) - z_p)), and RANGE instances the filter route cannot take: the segment sweep.
+//   k_sweep     the timeline is cut into time segments.  A CTA walks its segment in rounds: every row
+//               advances a cursor over the elements inside the round's time window (the rows are
+//               sorted, so the n-way merge is a set of cursors), attaches the payload the scan needs
+//               (next / delta + first flag) and appends it to a shared-memory batch.  A full batch is
+//               sorted into time order, scanned (prefix max of next / prefix sums of delta and flag)
+//               and evaluated.  Carry-ins at a segment start come from per-row binary searches, so
+//               segments are independent.
+//
+//   k_finalize  minimum over an instance's partial results, barrier, per-worker index recovery.
+//   k_trace     per-position intermediates of the steps for small instances (tests).
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>

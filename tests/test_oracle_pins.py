@@ -238,3 +238,34 @@ def test_trace_matches_the_selection():
         ws = tr["w_sum"]
         kmin = int(np.argmin(ws))
         assert ws[kmin] == w and tr["om_t"][kmin] == b
+
+
+# ------------------------------------------------------------------ the predictor (phase 1)
+def test_predictor_rows_are_arithmetic_from_the_last_timestamp():
+    rng = np.random.default_rng(21)
+    last = rng.integers(0, 10 ** 12, size=9)
+    iv = rng.integers(0, 10 ** 6, size=9)
+    out = o.predict(last, iv, 7)
+    assert out.shape == (9, 7)
+    assert (out[:, 0] == last + iv).all()
+    assert (np.diff(out, axis=1) == iv[:, None]).all()
+    with pytest.raises(ValueError):
+        o.predict([5], [-1], 3)
+    with pytest.raises(ValueError):
+        o.predict([2 ** 61], [2 ** 61], 3)
+
+
+def test_predictor_then_search_matches_the_common_period_closed_form():
+    # all workers predicted with one interval m: the best window misses only the largest circular gap of the phases
+    rng = np.random.default_rng(22)
+    for _ in range(100):
+        n, m, R = int(rng.integers(1, 9)), int(rng.integers(5, 400)), int(rng.integers(2, 9))
+        phase = rng.integers(0, m, size=n)
+        last = 10 ** 9 + phase                      # latest observed end of each worker
+        M = o.predict(last, np.full(n, m), R)
+        u = np.unique(phase)
+        gaps = np.diff(np.concatenate([u, [u[0] + m]]))
+        expect = 0 if len(u) == 1 else m - int(gaps.max())
+        w, b, idx = o.sweep(M, o.RANGE)
+        assert w == expect
+        assert (M[np.arange(n), idx] <= b).all() and M[np.arange(n), idx].max() == b
