@@ -42,7 +42,8 @@ typedef enum {
 
 enum {
     ZL_FLAG_CHECK_SORTED = 1,  /* verify every row is non-decreasing (one extra pass over the input) */
-    ZL_FLAG_FULL_SWEEP = 2     /* examine every timestamp even where the search could stop early    */
+    ZL_FLAG_FULL_SWEEP = 2,    /* examine every timestamp even where the search could stop early    */
+    ZL_FLAG_PREDICTOR = 4      /* the handle also holds a [max_batch][n][R] buffer for zl_predict_select_batched */
 };
 
 typedef struct {
@@ -91,6 +92,32 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out);
 zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B,
                             int32_t *d_idx, int64_t *d_barrier, int64_t *d_wait,
                             int32_t *d_status, void *cuda_stream);
+
+/*
+ * Phase 1 of ZipLine (Introduction; Section II, first property; Section III): the R future end
+ * timestamps of every worker are predicted from its most recent iteration interval under the
+ * stable-environment assumption.  The paper gives no formula; this is constant-interval
+ * extrapolation, e^p_i = last[p] + i * interval[p] for i = 1..R.
+ *
+ *   d_last      device, [B][n] int64: latest observed end timestamp of each worker, >= 0.
+ *   d_interval  device, [B][n] int64: its most recent iteration interval in microseconds, >= 0.
+ *   d_ts        device out, [B][n][R] int64, 16-byte aligned: the matrix zl_select_batched takes.
+ *
+ * A worker with a negative input gets a row of -1, one whose last prediction would reach 2^62 gets a
+ * row of 2^62; zl_select_batched reports ZL_ERR_INVALID_ARG for such an instance.  Asynchronous on
+ * cuda_stream; no handle, no scratch.
+ */
+zl_status zl_predict_batched(const int64_t *d_last, const int64_t *d_interval, int32_t B, int32_t n, int32_t R,
+                             int64_t *d_ts, void *cuda_stream);
+
+/*
+ * Both phases of ZipLine in one call: predict into the handle's own buffer (the handle must have been
+ * created with ZL_FLAG_PREDICTOR, else ZL_ERR_INVALID_ARG), then the search of zl_select_batched on it.
+ * Outputs, stream and error behaviour as for zl_select_batched.
+ */
+zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const int64_t *d_interval, int32_t B,
+                                    int32_t *d_idx, int64_t *d_barrier, int64_t *d_wait, int32_t *d_status,
+                                    void *cuda_stream);
 
 /*
  * The same search with HOST buffers (same shapes and meaning as above):

@@ -16,13 +16,14 @@ from . import build as _build
 ZL_OK = 0
 ZL_ERR_INVALID_ARG, ZL_ERR_UNSUPPORTED, ZL_ERR_NOMEM, ZL_ERR_CUDA, ZL_ERR_UNSORTED, ZL_ERR_TIMEOUT = range(1, 7)
 ZL_OBJ_RANGE, ZL_OBJ_SUM = 0, 1
-ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP = 1, 2
+ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP, ZL_FLAG_PREDICTOR = 1, 2, 4
 
 EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace_batched", "zl_destroy",
            "zl_set_option", "zl_status_string", "zl_workspace_bytes", "zl_launches_per_call",
            "zl_segments_per_instance", "zl_max_workers", "zl_trace_max_elements", "zl_last_cuda_error",
            "zl_profile_begin", "zl_profile_read", "zl_profile_end",
-           "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes", "zl_filter_counts")
+           "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes", "zl_filter_counts",
+           "zl_predict_batched", "zl_predict_select_batched")
 
 
 class zl_config(ctypes.Structure):
@@ -49,6 +50,10 @@ def _load() -> ctypes.CDLL:
     lib.zl_profile_begin.argtypes = [vp, i32]
     lib.zl_profile_read.argtypes = [vp, vp, vp]
     lib.zl_profile_end.argtypes = [vp]
+    lib.zl_predict_batched.argtypes = [vp, vp, i32, i32, i32, vp, vp]
+    lib.zl_predict_batched.restype = ctypes.c_int
+    lib.zl_predict_select_batched.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
+    lib.zl_predict_select_batched.restype = ctypes.c_int
     lib.zl_filter_counts.argtypes = [vp, i32, vp, vp, vp]
     lib.zl_filter_counts.restype = ctypes.c_int
     lib.zl_select_batched_noalloc.argtypes = [i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
@@ -137,6 +142,29 @@ class ZipLine:
         _check(rc, "zl_select_batched")
         return out
 
+    # -- zl_predict_select_batched -------------------------------------------------------
+    def predict_select_batched(self, last: torch.Tensor, interval: torch.Tensor, out: Selection | None = None,
+                               stream: torch.cuda.Stream | None = None) -> Selection:
+        """last, interval: CUDA int64 [B, n].  Needs a handle created with ZL_FLAG_PREDICTOR."""
+        B = last.shape[0]
+        if last.shape != (B, self.n) or interval.shape != (B, self.n):
+            raise ValueError(f"last and interval must be [B, {self.n}]")
+        if out is None:
+            dev = last.device
+            out = Selection(torch.empty((B, self.n), dtype=torch.int32, device=dev),
+                            torch.empty(B, dtype=torch.int64, device=dev),
+                            torch.empty(B, dtype=torch.int64, device=dev),
+                            torch.empty(B, dtype=torch.int32, device=dev))
+        s = stream if stream is not None else torch.cuda.current_stream(last.device)
+        rc = lib.zl_predict_select_batched(self._h, _dev_ptr(last, torch.int64, B * self.n, "last"),
+                                           _dev_ptr(interval, torch.int64, B * self.n, "interval"), B,
+                                           _dev_ptr(out.idx, torch.int32, B * self.n, "idx"),
+                                           _dev_ptr(out.barrier, torch.int64, B, "barrier"),
+                                           _dev_ptr(out.wait, torch.int64, B, "wait"),
+                                           _dev_ptr(out.status, torch.int32, B, "status"), s.cuda_stream)
+        _check(rc, "zl_predict_select_batched")
+        return out
+
     # -- zl_select_batched_host ----------------------------------------------------------
     def select_batched_host(self, ts: torch.Tensor, out: Selection | None = None) -> Selection:
         """ts: host int64 [B, n, R] (pinned for speed).  Returns host tensors; synchronous."""
@@ -199,6 +227,18 @@ class ZipLine:
             self.destroy()
         except Exception:
             pass
+
+
+def zl_predict_batched(last: torch.Tensor, interval: torch.Tensor, R: int,
+                       stream: torch.cuda.Stream | None = None) -> torch.Tensor:
+    """Phase 1 of ZipLine: CUDA int64 [B, n] last end timestamps and intervals -> [B, n, R] predictions."""
+    B, n = last.shape
+    out = torch.empty((B, n, R), dtype=torch.int64, device=last.device)
+    s = stream if stream is not None else torch.cuda.current_stream(last.device)
+    rc = lib.zl_predict_batched(_dev_ptr(last, torch.int64, B * n, "last"), _dev_ptr(interval, torch.int64, B * n, "interval"),
+                                B, n, R, out.data_ptr(), s.cuda_stream)
+    _check(rc, "zl_predict_batched")
+    return out
 
 
 def zl_noalloc_max_batch() -> int:

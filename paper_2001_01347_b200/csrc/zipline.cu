@@ -1131,6 +1131,28 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
     }
 }
 
+// ------------------------------------------------------------------------------ predictor
+// One CTA per row: e_i = last + i * interval, i = 1..R, written with 16-byte stores where the row allows.
+__global__ void __launch_bounds__(256) k_predict(const int64_t *last, const int64_t *interval, int R, int64_t *ts) {
+    const size_t row = blockIdx.x;
+    const int64_t l = ldg64(last + row), iv = ldg64(interval + row);
+    int64_t *out = ts + row * (size_t)R;
+    int64_t base = l, step = iv;
+    if (l < 0 || iv < 0) { base = -1; step = 0; }                 // marks the instance invalid for the search
+    else if (__umul64hi((uint64_t)R, (uint64_t)iv) != 0 || (uint64_t)R * (uint64_t)iv >= (uint64_t)VALUE_LIMIT ||
+             (uint64_t)l + (uint64_t)R * (uint64_t)iv >= (uint64_t)VALUE_LIMIT) { base = VALUE_LIMIT; step = 0; }
+    if ((R & 1) == 0 && (((uintptr_t)out) & 15) == 0) {
+        for (int i = 2 * threadIdx.x; i < R; i += 2 * blockDim.x) {
+            longlong2 v;
+            v.x = base + (int64_t)(i + 1) * step;
+            v.y = base + (int64_t)(i + 2) * step;
+            *reinterpret_cast<longlong2 *>(out + i) = v;
+        }
+    } else {
+        for (int i = threadIdx.x; i < R; i += blockDim.x) out[i] = base + (int64_t)(i + 1) * step;
+    }
+}
+
 // ------------------------------------------------------------------------------ trace
 struct TKey {
     uint64_t t; uint32_t f, pad;
@@ -1216,6 +1238,7 @@ struct zl_handle {
     int num_sms;
     zl::InstMeta *d_meta;
     zl::SegResult *d_seg;
+    int64_t *d_pred;         // ZL_FLAG_PREDICTOR: predicted timestamps, [max_batch][n][R]
     zl::FilterBufs fb;       // RANGE: buffers of the filter route (device), sized for max_batch
     int nres;                // SegResult slots per instance
     size_t ws_bytes;
@@ -1399,7 +1422,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     *out = nullptr;
     if (cfg->n_workers < 1 || cfg->lookahead_R < 1 || cfg->max_batch < 1) return ZL_ERR_INVALID_ARG;
     if (cfg->objective != ZL_OBJ_RANGE && cfg->objective != ZL_OBJ_SUM) return ZL_ERR_INVALID_ARG;
-    if (cfg->flags & ~(ZL_FLAG_CHECK_SORTED | ZL_FLAG_FULL_SWEEP)) return ZL_ERR_INVALID_ARG;
+    if (cfg->flags & ~(ZL_FLAG_CHECK_SORTED | ZL_FLAG_FULL_SWEEP | ZL_FLAG_PREDICTOR)) return ZL_ERR_INVALID_ARG;
     if (cfg->n_workers > zl::MAX_WORKERS) return ZL_ERR_UNSUPPORTED;
     if ((long long)cfg->n_workers * cfg->lookahead_R > (1LL << 31) - 1) return ZL_ERR_UNSUPPORTED;
     if (cfg->max_batch > 65535) return ZL_ERR_UNSUPPORTED;
@@ -1438,16 +1461,18 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     const size_t seg_b = (size_t)cfg->max_batch * h->nres * sizeof(zl::SegResult);
     if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_meta, meta_b);
     if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_seg, seg_b);
+    const size_t pred_b = (cfg->flags & ZL_FLAG_PREDICTOR) ? (size_t)cfg->max_batch * cfg->n_workers * cfg->lookahead_R * 8 : 0;
+    if (e == cudaSuccess && pred_b) e = cudaMalloc((void **)&h->d_pred, pred_b);
     if (e == cudaSuccess) e = raise_shared_memory_limits();   // more than the default 48 KB of dynamic shared memory
     if (e != cudaSuccess) {
         zl_status st = cuda_fail(nullptr, e);
-        cudaFree(h->d_meta); cudaFree(h->d_seg);
+        cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
         cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
         cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
         delete h;
         return st;
     }
-    h->ws_bytes = meta_b + seg_b + filter_b;
+    h->ws_bytes = meta_b + seg_b + filter_b + pred_b;
     *out = h;
     return ZL_OK;
 }
@@ -1503,7 +1528,7 @@ zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_stage) {
 zl_status zl_destroy(zl_handle *h) {
     if (!h) return ZL_OK;
     cudaSetDevice(h->cfg.device);
-    cudaFree(h->d_meta); cudaFree(h->d_seg);
+    cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
     cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
     cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
     cudaFree(h->s_ts); cudaFree(h->s_idx); cudaFree(h->s_barrier); cudaFree(h->s_wait); cudaFree(h->s_status);
@@ -1595,6 +1620,27 @@ zl_status zl_filter_counts(zl_handle *h, int32_t B, uint32_t *h_filtered, uint32
             ZL_CUDA(h, cudaMemcpy2D(dst[i], sizeof(uint32_t), (const char *)h->d_meta + off[i], sizeof(zl::InstMeta),
                                     sizeof(uint32_t), (size_t)B, cudaMemcpyDeviceToHost));
     return ZL_OK;
+}
+
+zl_status zl_predict_batched(const int64_t *d_last, const int64_t *d_interval, int32_t B, int32_t n, int32_t R,
+                             int64_t *d_ts, void *cuda_stream) {
+    if (!d_last || !d_interval || !d_ts || B < 1 || n < 1 || R < 1) return ZL_ERR_INVALID_ARG;
+    if (((uintptr_t)d_last & 7) || ((uintptr_t)d_interval & 7) || ((uintptr_t)d_ts & 15)) return ZL_ERR_INVALID_ARG;
+    if ((long long)B * n > 0x7fffffffLL) return ZL_ERR_UNSUPPORTED;
+    const int threads = std::max(32, std::min(256, pow2_ceil((R + 1) / 2)));
+    zl::k_predict<<<(unsigned)((long long)B * n), threads, 0, (cudaStream_t)cuda_stream>>>(d_last, d_interval, R, d_ts);
+    return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;
+}
+
+zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const int64_t *d_interval, int32_t B,
+                                    int32_t *d_idx, int64_t *d_barrier, int64_t *d_wait, int32_t *d_status,
+                                    void *cuda_stream) {
+    if (!h || !h->d_pred) return ZL_ERR_INVALID_ARG;
+    if (B < 1 || B > h->cfg.max_batch) return ZL_ERR_INVALID_ARG;
+    zl_status rc = zl_predict_batched(d_last, d_interval, B, h->cfg.n_workers, h->cfg.lookahead_R, h->d_pred, cuda_stream);
+    if (rc != ZL_OK) return rc;
+    ++h->launches;
+    return zl_select_batched(h, h->d_pred, B, d_idx, d_barrier, d_wait, d_status, cuda_stream);
 }
 
 zl_status zl_select_batched_host(zl_handle *h, const int64_t *h_ts, int32_t B, int32_t *h_idx, int64_t *h_barrier,
