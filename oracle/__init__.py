@@ -49,6 +49,8 @@ def _load():
         lib.zlo_alg2.restype = ci
         lib.zlo_trace.argtypes = [vp, ci, ci] + [vp] * 11
         lib.zlo_trace.restype = ci
+        lib.zlo_gridscan.argtypes = [vp, ci, ci, ci, vp, vp, vp]
+        lib.zlo_gridscan.restype = ci
         lib.zlo_predict.argtypes = [vp, vp, ci, ci, vp]
         lib.zlo_predict.restype = ci
         _lib = lib
@@ -116,6 +118,17 @@ def trace(M) -> dict:
     out = {k: np.empty(n * R, dtype=dt) for k, dt in TRACE_FIELDS}
     _check(_load().zlo_trace(M.ctypes.data, n, R, *[out[k].ctypes.data for k, _ in TRACE_FIELDS]))
     return out
+
+
+def gridscan(M, full: bool = False):
+    """Algorithm 1 (GridScan), or FullGridScan with full=True -> (wait, barrier, idx of Z*). Heuristic baselines."""
+    M = _matrix(M)
+    n, R = M.shape
+    wait, barrier = ctypes.c_int64(), ctypes.c_int64()
+    idx = np.empty(n, dtype=np.int32)
+    _check(_load().zlo_gridscan(M.ctypes.data, n, R, int(bool(full)), ctypes.addressof(wait),
+                                ctypes.addressof(barrier), idx.ctypes.data))
+    return int(wait.value), int(barrier.value), idx
 
 
 def predict(last, interval, R: int) -> np.ndarray:

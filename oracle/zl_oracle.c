@@ -33,6 +33,7 @@
  *                     the O(n) evaluation is too slow
  *   zlo_alg2          Algorithm 2 step by step (drop min(Z), refill until |Z|=n)
  *   zlo_trace         per-position intermediates of the pass, for kernel tests
+ *   zlo_gridscan      Algorithm 1 (GridScan) and its rotation over all rows (FullGridScan): the paper's baselines
  *   zlo_predict       phase 1 of ZipLine: R future end timestamps per worker from its most recent interval
  *
  * Return codes: 0 ok, -1 bad argument, -2 a row is not non-decreasing,
@@ -334,5 +335,54 @@ int zlo_predict(const int64_t *last, const int64_t *interval, int n, int R, int6
             out[(size_t)p * R + (i - 1)] = (int64_t)v;
         }
     }
+    return 0;
+}
+
+/* ------------------------------------------------------- Algorithm 1 (GridScan) / FullGridScan
+ * GridScan (Section IV, Algorithm 1): the designated row is the one with the earliest first element
+ * (the lowest-numbered such row).  For every point e of the designated row, Z holds e and, from every
+ * other row, the point at the shortest distance |M[p][i] - e|; d_Z = max(Z) - min(Z); the first Z with
+ * a strictly smaller d_Z is kept.  FullGridScan (same section) designates every row in turn, rows in
+ * order, keeping the strict minimum over all n*R candidates.
+ * Readings: between two points of a row at equal distance the earlier one is taken; among equal points
+ * of a row the one with the lowest index.  Heuristics: wait >= the optimum of the search above.
+ * idx[p] = index of the element of Z* in row p; barrier = max(Z*). */
+int zlo_gridscan(const int64_t *M, int n, int R, int full, int64_t *wait, int64_t *barrier, int32_t *idx) {
+    if (!M || n < 1 || R < 1 || !wait || !barrier || !idx) return -1;
+    int rc = check_rows(M, n, R);
+    if (rc) return rc;
+    int32_t *z = (int32_t *)malloc((size_t)n * sizeof(int32_t));
+    if (!z) return -4;
+    int pb = 0;
+    for (int p = 1; p < n; ++p) if (M[(size_t)p * R] < M[(size_t)pb * R]) pb = p;
+    int have = 0;
+    int64_t best = 0, best_max = 0;
+    for (int q = full ? 0 : pb; q < (full ? n : pb + 1); ++q) {
+        for (int j = 0; j < R; ++j) {
+            const int64_t e = M[(size_t)q * R + j];
+            int64_t mx = e, mn = e;
+            for (int p = 0; p < n; ++p) {
+                if (p == q) { z[p] = j; continue; }
+                int bi = 0;
+                int64_t bd = INT64_MAX;
+                for (int i = 0; i < R; ++i) {                     /* shortest distance; earlier point on ties */
+                    int64_t v = M[(size_t)p * R + i];
+                    int64_t dist = v > e ? v - e : e - v;
+                    if (dist < bd) { bd = dist; bi = i; }
+                }
+                z[p] = bi;
+                int64_t v = M[(size_t)p * R + bi];
+                if (v > mx) mx = v;
+                if (v < mn) mn = v;
+            }
+            if (!have || mx - mn < best) {
+                have = 1; best = mx - mn; best_max = mx;
+                memcpy(idx, z, (size_t)n * sizeof(int32_t));
+            }
+        }
+    }
+    free(z);
+    *wait = best;
+    *barrier = best_max;
     return 0;
 }

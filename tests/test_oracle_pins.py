@@ -269,3 +269,52 @@ def test_predictor_then_search_matches_the_common_period_closed_form():
         w, b, idx = o.sweep(M, o.RANGE)
         assert w == expect
         assert (M[np.arange(n), idx] <= b).all() and M[np.arange(n), idx].max() == b
+
+
+# ------------------------------------------------------------------ Algorithm 1 (GridScan) and FullGridScan
+def gridscan_python(M, full):
+    """Algorithm 1 written out from the listing: nearest point of every other row to each designated point."""
+    n, R = len(M), len(M[0])
+    pb = min(range(n), key=lambda p: (M[p][0], p))
+    best = None
+    for q in (range(n) if full else [pb]):
+        for j in range(R):
+            e = M[q][j]
+            z = []
+            for p in range(n):
+                if p == q:
+                    z.append(j)
+                else:
+                    z.append(min(range(R), key=lambda i: (abs(M[p][i] - e), i)))
+            vals = [M[p][z[p]] for p in range(n)]
+            d = max(vals) - min(vals)
+            if best is None or d < best[0]:
+                best = (d, max(vals), z)
+    return best
+
+
+@pytest.mark.parametrize("full", [False, True])
+@pytest.mark.parametrize("regime", ["dense", "sparse", "strict"])
+def test_gridscan_matches_the_listing_and_never_beats_the_optimum(full, regime):
+    rng = np.random.default_rng(400 + full + len(regime))
+    misses = 0
+    for _ in range(300):
+        M = random_instance(rng, regime)
+        w, b, idx = o.gridscan(M, full)
+        assert (w, b, list(idx)) == gridscan_python(M.tolist(), full)
+        chosen = M[np.arange(M.shape[0]), idx]
+        assert chosen.max() - chosen.min() == w and chosen.max() == b
+        opt = o.sweep(M, o.RANGE)[0]
+        assert w >= opt
+        misses += w > opt
+    if full and regime != "dense":
+        assert misses < 300                     # FullGridScan finds the optimum at least sometimes
+
+
+def test_fullgridscan_is_never_worse_than_gridscan():
+    rng = np.random.default_rng(77)
+    for _ in range(200):
+        M = random_instance(rng, "strict")
+        assert o.gridscan(M, True)[0] <= o.gridscan(M, False)[0]
+    # a hand case: rows [0,10,20], [4,14,24], [9,19,29]; designated row 0; e=0 -> {0,4,9} d=9; e=10 -> {10,14,9} d=5
+    assert o.gridscan([[0, 10, 20], [4, 14, 24], [9, 19, 29]])[:2] == (5, 14)
