@@ -120,6 +120,24 @@ zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const i
                                     void *cuda_stream);
 
 /*
+ * The paper's baselines (Section IV, Algorithm 1): GridScan designates the row with the earliest first
+ * timestamp and, for each of its R points, takes from every other row the point at the shortest distance;
+ * FullGridScan (full != 0) designates every row in turn (n*R candidate sets).  The candidate with the
+ * smallest max(Z) - min(Z) wins, the first one on ties.  Heuristics: the result is never below
+ * zl_select_batched's.  Readings: of two points of a row at equal distance the earlier one is taken, of
+ * equal points the one with the lowest index.
+ *
+ *   d_ts       device, [B][n][R] int64, rows non-decreasing (as for zl_select_batched; not checked here).
+ *   d_scratch  device, int64, B*R elements (B*n*R when full): the candidates' d_Z; contents undefined after.
+ *   d_idx      device out, [B][n] int32: index of the element of Z* in each row.
+ *   d_barrier, d_wait  device out, [B] int64: max(Z*) and max(Z*) - min(Z*).
+ * Asynchronous on cuda_stream; no handle.
+ */
+zl_status zl_gridscan_batched(const int64_t *d_ts, int32_t B, int32_t n, int32_t R, int32_t full,
+                              int64_t *d_scratch, int32_t *d_idx, int64_t *d_barrier, int64_t *d_wait,
+                              void *cuda_stream);
+
+/*
  * The same search with HOST buffers (same shapes and meaning as above):
  * copies the input to the device, runs the kernels, copies the results back
  * and waits for them.  Staging buffers are allocated by the first such call

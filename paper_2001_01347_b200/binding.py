@@ -23,7 +23,7 @@ EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace
            "zl_segments_per_instance", "zl_max_workers", "zl_trace_max_elements", "zl_last_cuda_error",
            "zl_profile_begin", "zl_profile_read", "zl_profile_end",
            "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes", "zl_filter_counts",
-           "zl_predict_batched", "zl_predict_select_batched")
+           "zl_predict_batched", "zl_predict_select_batched", "zl_gridscan_batched")
 
 
 class zl_config(ctypes.Structure):
@@ -50,6 +50,8 @@ def _load() -> ctypes.CDLL:
     lib.zl_profile_begin.argtypes = [vp, i32]
     lib.zl_profile_read.argtypes = [vp, vp, vp]
     lib.zl_profile_end.argtypes = [vp]
+    lib.zl_gridscan_batched.argtypes = [vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.zl_gridscan_batched.restype = ctypes.c_int
     lib.zl_predict_batched.argtypes = [vp, vp, i32, i32, i32, vp, vp]
     lib.zl_predict_batched.restype = ctypes.c_int
     lib.zl_predict_select_batched.argtypes = [vp, vp, vp, i32, vp, vp, vp, vp, vp]
@@ -239,6 +241,22 @@ def zl_predict_batched(last: torch.Tensor, interval: torch.Tensor, R: int,
                                 B, n, R, out.data_ptr(), s.cuda_stream)
     _check(rc, "zl_predict_batched")
     return out
+
+
+def zl_gridscan_batched(ts: torch.Tensor, full: bool = False, stream: torch.cuda.Stream | None = None):
+    """The paper's heuristic baselines (Algorithm 1): GridScan, or FullGridScan with full=True.
+    ts: CUDA int64 [B, n, R] -> (idx [B, n] int32, barrier [B], wait [B])."""
+    B, n, R = ts.shape
+    dev = ts.device
+    scratch = torch.empty(B * (n * R if full else R), dtype=torch.int64, device=dev)
+    idx = torch.empty((B, n), dtype=torch.int32, device=dev)
+    barrier = torch.empty(B, dtype=torch.int64, device=dev)
+    wait = torch.empty(B, dtype=torch.int64, device=dev)
+    s = stream if stream is not None else torch.cuda.current_stream(dev)
+    rc = lib.zl_gridscan_batched(_dev_ptr(ts, torch.int64, B * n * R, "ts"), B, n, R, int(bool(full)),
+                                 scratch.data_ptr(), idx.data_ptr(), barrier.data_ptr(), wait.data_ptr(), s.cuda_stream)
+    _check(rc, "zl_gridscan_batched")
+    return idx, barrier, wait
 
 
 def zl_noalloc_max_batch() -> int:

@@ -1131,6 +1131,100 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
     }
 }
 
+// ------------------------------------------------------------------------------ GridScan / FullGridScan
+// Value of the point of a sorted row at the shortest distance from e (the earlier one on ties).
+__device__ __forceinline__ int64_t nearest_value(const int64_t *row, int R, int64_t e) {
+    int lo = 0, hi = R;                           // first index with row[i] >= e
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (ldg64(row + mid) < e) lo = mid + 1; else hi = mid;
+    }
+    if (lo == 0) return ldg64(row);
+    const int64_t left = ldg64(row + lo - 1);
+    if (lo == R) return left;
+    const int64_t right = ldg64(row + lo);
+    return e - left <= right - e ? left : right;
+}
+
+// Lowest index of a sorted row that holds value v (v occurs in the row).
+__device__ __forceinline__ int first_index_of(const int64_t *row, int R, int64_t v) {
+    int lo = 0, hi = R;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (ldg64(row + mid) < v) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// Row with the earliest first timestamp (lowest-numbered on ties); every thread of the block gets it.
+__device__ int designated_row(const int64_t *inst, int n, int R, uint64_t *tmp) {
+    uint64_t best = ~0ull;                         // (first timestamp, row) packed: timestamps are below 2^62
+    uint64_t bestp = 0;
+    for (int p = threadIdx.x; p < n; p += blockDim.x) {
+        const uint64_t v = (uint64_t)ldg64(inst + (size_t)p * R);
+        if (v < best) { best = v; bestp = (uint64_t)p; }
+    }
+    uint64_t tot;
+    block_scan_excl<uint64_t>(best, OpMin(), ~0ull, tmp, &tot);
+    uint64_t cand = best == tot ? bestp : ~0ull, totp;
+    block_scan_excl<uint64_t>(cand, OpMin(), ~0ull, tmp, &totp);
+    return (int)totp;
+}
+
+// d_Z of one candidate per CTA.  grid (candidates, B); candidate c = designated point (row c / R, index c % R)
+// when full, else point c of the designated row.
+__global__ void __launch_bounds__(256) k_gridscan_eval(const int64_t *ts, int n, int R, int full, int64_t *cand) {
+    __shared__ uint64_t tmp[34];
+    const int b = blockIdx.y, c = blockIdx.x;
+    const int64_t *inst = ts + (size_t)b * n * R;
+    const int q = full ? c / R : designated_row(inst, n, R, tmp);
+    const int j = full ? c % R : c;
+    const int64_t e = ldg64(inst + (size_t)q * R + j);
+    uint64_t mx = (uint64_t)e, mn = (uint64_t)e;
+    for (int p = threadIdx.x; p < n; p += blockDim.x) {
+        if (p == q) continue;
+        const uint64_t v = (uint64_t)nearest_value(inst + (size_t)p * R, R, e);
+        mx = max(mx, v); mn = min(mn, v);
+    }
+    uint64_t gmx, gmn;
+    block_scan_excl<uint64_t>(mx, OpMax(), 0ull, tmp, &gmx);
+    block_scan_excl<uint64_t>(mn, OpMin(), ~0ull, tmp, &gmn);
+    if (threadIdx.x == 0) cand[(size_t)b * gridDim.x + c] = (int64_t)(gmx - gmn);
+}
+
+// First minimal candidate of an instance, then its Z*.  grid B
+__global__ void __launch_bounds__(256) k_gridscan_pick(const int64_t *ts, int n, int R, int full, int ncand, const int64_t *cand,
+                                                       int32_t *idx, int64_t *barrier, int64_t *wait) {
+    __shared__ uint64_t tmp[34];
+    const int b = blockIdx.x;
+    const int64_t *inst = ts + (size_t)b * n * R;
+    uint64_t bd = ~0ull, bc = ~0ull;
+    for (int c = threadIdx.x; c < ncand; c += blockDim.x) {
+        const uint64_t d = (uint64_t)cand[(size_t)b * ncand + c];
+        if (d < bd) { bd = d; bc = (uint64_t)c; }                 // a thread sees its candidates in ascending order
+    }
+    uint64_t gd, gc;
+    block_scan_excl<uint64_t>(bd, OpMin(), ~0ull, tmp, &gd);
+    block_scan_excl<uint64_t>(bd == gd ? bc : ~0ull, OpMin(), ~0ull, tmp, &gc);
+    const int c = (int)gc;
+    const int q = full ? c / R : designated_row(inst, n, R, tmp);
+    const int j = full ? c % R : c;
+    const int64_t e = ldg64(inst + (size_t)q * R + j);
+    uint64_t mx = (uint64_t)e;
+    for (int p = threadIdx.x; p < n; p += blockDim.x) {
+        int res = j;
+        if (p != q) {
+            const int64_t v = nearest_value(inst + (size_t)p * R, R, e);
+            res = first_index_of(inst + (size_t)p * R, R, v);
+            mx = max(mx, (uint64_t)v);
+        }
+        idx[(size_t)b * n + p] = res;
+    }
+    uint64_t gmx;
+    block_scan_excl<uint64_t>(mx, OpMax(), 0ull, tmp, &gmx);
+    if (threadIdx.x == 0) { barrier[b] = (int64_t)gmx; wait[b] = (int64_t)gd; }
+}
+
 // ------------------------------------------------------------------------------ predictor
 // One CTA per row: e_i = last + i * interval, i = 1..R, written with 16-byte stores where the row allows.
 __global__ void __launch_bounds__(256) k_predict(const int64_t *last, const int64_t *interval, int R, int64_t *ts) {
@@ -1620,6 +1714,19 @@ zl_status zl_filter_counts(zl_handle *h, int32_t B, uint32_t *h_filtered, uint32
             ZL_CUDA(h, cudaMemcpy2D(dst[i], sizeof(uint32_t), (const char *)h->d_meta + off[i], sizeof(zl::InstMeta),
                                     sizeof(uint32_t), (size_t)B, cudaMemcpyDeviceToHost));
     return ZL_OK;
+}
+
+zl_status zl_gridscan_batched(const int64_t *d_ts, int32_t B, int32_t n, int32_t R, int32_t full, int64_t *d_scratch,
+                              int32_t *d_idx, int64_t *d_barrier, int64_t *d_wait, void *cuda_stream) {
+    if (!d_ts || !d_scratch || !d_idx || !d_barrier || !d_wait || B < 1 || n < 1 || R < 1) return ZL_ERR_INVALID_ARG;
+    if (B > 65535) return ZL_ERR_UNSUPPORTED;
+    const long long ncand = full ? (long long)n * R : R;
+    if (ncand > 0x7fffffffLL) return ZL_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int threads = std::max(32, std::min(256, pow2_ceil(n)));
+    zl::k_gridscan_eval<<<dim3((unsigned)ncand, B), threads, 0, st>>>(d_ts, n, R, full ? 1 : 0, d_scratch);
+    zl::k_gridscan_pick<<<B, 256, 0, st>>>(d_ts, n, R, full ? 1 : 0, (int)ncand, d_scratch, d_idx, d_barrier, d_wait);
+    return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;
 }
 
 zl_status zl_predict_batched(const int64_t *d_last, const int64_t *d_interval, int32_t B, int32_t n, int32_t R,
