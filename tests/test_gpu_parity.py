@@ -272,3 +272,17 @@ def test_mixed_batch_of_routes():
     sel, filtered, refined, overflow = _routes(ts)
     assert overflow.tolist() == [0, 0, 1, 0, 0]
     assert_same(ts, 0, (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()))
+
+
+# ---------------------------------------------------------------- extreme shapes
+@pytest.mark.parametrize("objective", OBJ)
+def test_extreme_aspect_ratios(objective):
+    rng = np.random.default_rng(900 + objective)
+    nmax = zl.zl_max_workers()
+    for n, R, B, hi in ((nmax, 3, 2, 1000), (nmax, 1, 1, 50), (2, 50_000, 2, 100), (1, 100_000, 1, 7),
+                        (3000, 7, 2, 10 ** 5), (5, 4097, 3, 10 ** 4)):
+        inc = rng.integers(0, hi, size=(B, n, R))
+        ts = (rng.integers(0, 3 * hi, size=(B, n, 1)) + np.cumsum(inc, axis=2)).astype(np.int64)
+        assert_same(ts, objective, gpu_select(ts, objective))
+    with pytest.raises(zl.ZipLineError):
+        zl.ZipLine(nmax + 1, 2, 1, objective)
