@@ -273,8 +273,8 @@ __global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, 
 // 64 timestamps in flight per warp), tests every element against the table and appends the survivors,
 // as (T << 32 | next), to the region's list; the per-cell maximum of `next` over the survivors goes to
 // cellmax for the refinement.  Rows whose length is odd, or a misaligned base, take 8-byte copies.
-constexpr int FILTER_STAGES = 4;      // ring slots per warp
-constexpr int FILTER_CHUNK = 128;     // timestamps per slot (two 16-byte copies per lane)
+constexpr int FILTER_STAGES = 3;      // ring slots per warp
+constexpr int FILTER_CHUNK = 256;     // timestamps per slot (FILTER_CHUNK / 64 16-byte copies per lane)
 constexpr int FILTER_SLOT = FILTER_CHUNK + 2;   // + the successor of the slot's last element, + padding
 
 __device__ __forceinline__ void cp_async16(void *smem, const void *gmem) {
@@ -334,16 +334,33 @@ __device__ __forceinline__ void filter_pair(const FilterCtx &c, int lane, bool v
 // The 64 elements of a slot starting at `off`: element pairs per lane, successor of the pair from the
 // slot itself (the element after the slot's last one sits right behind it).  Returns the time of the
 // last valid element handled by lane 31 (0xffffffff past the row's end).
-__device__ __forceinline__ uint32_t filter_half(const FilterCtx &C, const int64_t *slot, int off, int i0, int R,
+__device__ __forceinline__ uint32_t filter_half(const FilterCtx &C, const int64_t *slot, int off, int i0, int lim, int R,
                                                 uint32_t tminlo, int lane) {
     const int i = i0 + off + 2 * lane;
-    const bool va = i < R, vb = i + 1 < R;
+    const bool va = i < lim, vb = i + 1 < lim;                    // lim: end of what was requested of the row (<= R)
     const longlong2 ab = *reinterpret_cast<const longlong2 *>(slot + off + 2 * lane);
     const uint32_t Ta = va ? (uint32_t)(uint64_t)ab.x - tminlo : 0xffffffffu;
     const uint32_t Tb = vb ? (uint32_t)(uint64_t)ab.y - tminlo : 0xffffffffu;
     const uint32_t nb = i + 2 < R ? (uint32_t)(uint64_t)slot[off + 2 * lane + 2] - tminlo : 0xffffffffu;
     filter_pair(C, lane, va, Ta, Tb, vb, Tb, nb);
     return __shfl_sync(FULL, Tb, 31);
+}
+
+// 128 timestamps of a slot, with the one after them, that lie inside the row: no bounds checks, one vote
+// for all four elements of a lane.  Returns the time of the last of the 128.
+__device__ __forceinline__ uint32_t filter_slot_inside(const FilterCtx &C, const int64_t *slot, uint32_t tminlo, int lane) {
+    const longlong2 p0 = *reinterpret_cast<const longlong2 *>(slot + 2 * lane);
+    const longlong2 p1 = *reinterpret_cast<const longlong2 *>(slot + 64 + 2 * lane);
+    const uint32_t a0 = (uint32_t)(uint64_t)p0.x - tminlo, b0 = (uint32_t)(uint64_t)p0.y - tminlo;
+    const uint32_t a1 = (uint32_t)(uint64_t)p1.x - tminlo, b1 = (uint32_t)(uint64_t)p1.y - tminlo;
+    const uint32_t n0 = (uint32_t)(uint64_t)slot[2 * lane + 2] - tminlo, n1 = (uint32_t)(uint64_t)slot[64 + 2 * lane + 2] - tminlo;
+    const bool k = (a0 <= C.lmin && b0 - a0 > C.dmin) || (b0 <= C.lmin && n0 - b0 > C.dmin) ||
+                   (a1 <= C.lmin && b1 - a1 > C.dmin) || (b1 <= C.lmin && n1 - b1 > C.dmin);
+    if (__any_sync(FULL, k)) {                                   // rare: some element may pass the table
+        filter_pair(C, lane, true, a0, b0, true, b0, n0);
+        filter_pair(C, lane, true, a1, b1, true, b1, n1);
+    }
+    return __shfl_sync(FULL, b1, 31);
 }
 
 __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R, int flags, int rows_per_cta,
@@ -370,15 +387,14 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
     C.cscale = M.cscale; C.fscale = M.fscale; C.lmin = lmin; C.regcap = (uint32_t)F.regcap; C.dmin = M.dmin;
     const int r0 = blockIdx.x * rows_per_cta, r1 = min(r0 + rows_per_cta, n);
     const bool vec2 = (R % 2 == 0) && (((uintptr_t)ts & 15) == 0);
-    const int nchunks = (R + FILTER_CHUNK - 1) / FILTER_CHUNK;
     const size_t rstride = (size_t)nw * R;                        // between consecutive rows of this warp
 
-    // this warp's rows, in rounds of up to 32: lane j holds the request (in slots) of the round's j-th row
+    // this warp's rows, in rounds of up to 32: lane j holds the request of the round's j-th row, i.e. how many of
+    // its leading timestamps are copied through the ring (a multiple of 64, or R)
     for (int rbase = r0 + warp; rbase < r1; rbase += 32 * nw) {
         const int nrows = min(32, (r1 - rbase + nw - 1) / nw);
         int req = 0;
-        if (lane < nrows)
-            req = full ? nchunks : min(nchunks, (int)((F.rowhint[(size_t)b * n + rbase + lane * nw] + FILTER_CHUNK - 1) / FILTER_CHUNK));
+        if (lane < nrows) req = full ? R : min(R, (int)((F.rowhint[(size_t)b * n + rbase + lane * nw] + 63) & ~63u));
         const int64_t *row_i = ts + ((size_t)b * n + rbase) * R, *row_p = row_i;
         int ji = 0, ci = 0, jp = 0, cp = 0, inflight = 0, slot_i = 0, slot_p = 0;
         int req_i = __shfl_sync(FULL, req, 0), req_p = req_i;
@@ -386,43 +402,59 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
         while (jp < nrows) {
             while (inflight < FILTER_STAGES && ji < nrows) {
                 int64_t *slot = ring + (size_t)slot_i * FILTER_SLOT;
-                const int i = ci * FILTER_CHUNK + 2 * lane;
+                const int base = ci * FILTER_CHUNK;
+                const int i = base + 2 * lane;
                 if (vec2) {
-                    if (i < R) cp_async16(slot + 2 * lane, row_i + i);
-                    if (i + 64 < R) cp_async16(slot + 64 + 2 * lane, row_i + i + 64);
+#pragma unroll
+                    for (int k = 0; k < FILTER_CHUNK / 64; ++k)
+                        if (i + 64 * k < req_i) cp_async16(slot + 64 * k + 2 * lane, row_i + i + 64 * k);
                 } else {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) {
+                    for (int k = 0; k < FILTER_CHUNK / 32; ++k) {
                         const int e = i + (k >> 1) * 64 + (k & 1);
-                        if (e < R) cp_async8(slot + (k >> 1) * 64 + 2 * lane + (k & 1), row_i + e);
+                        if (e < req_i) cp_async8(slot + (k >> 1) * 64 + 2 * lane + (k & 1), row_i + e);
                     }
                 }
-                if (lane == 31 && i + 66 < R) cp_async8(slot + FILTER_CHUNK, row_i + i + 66);   // successor of the slot's last element
+                // the element after the last one copied into this slot (its successor)
+                const int endi = min(base + FILTER_CHUNK, req_i);
+                if (lane == 31 && endi < R) cp_async8(slot + (endi - base), row_i + endi);
                 cp_async_commit();
                 ++inflight;
                 slot_i = slot_i + 1 == FILTER_STAGES ? 0 : slot_i + 1;
-                if (++ci == req_i) {
+                if (endi == req_i) {
                     ci = 0; ++ji; row_i += rstride;
                     req_i = __shfl_sync(FULL, req, min(ji, 31));
+                } else {
+                    ++ci;
                 }
             }
             cp_async_wait_pending(inflight - 1);
             __syncwarp();
+            const int i0 = cp * FILTER_CHUNK;
+            const int L = min(FILTER_CHUNK, req_p - i0);           // timestamps of the row in this slot
             if (!finished) {
                 const int64_t *slot = ring + (size_t)slot_p * FILTER_SLOT;
-                const int i0 = cp * FILTER_CHUNK;
-                uint32_t lastT = filter_half(C, slot, 0, i0, R, tminlo, lane);
-                if (full || lastT <= lmin) lastT = filter_half(C, slot, 64, i0, R, tminlo, lane);
+                uint32_t lastT = 0;
+#pragma unroll
+                for (int sub = 0; sub < FILTER_CHUNK; sub += 128) {
+                    if (sub >= L || (sub && !full && lastT > lmin)) break;   // rows are sorted: the rest is past lmin
+                    if (sub + 128 <= L && i0 + sub + 128 < R) {
+                        lastT = filter_slot_inside(C, slot + sub, tminlo, lane);
+                    } else {
+                        lastT = filter_half(C, slot, sub, i0, req_p, R, tminlo, lane);
+                        if (sub + 64 < L && (full || lastT <= lmin)) lastT = filter_half(C, slot, sub + 64, i0, req_p, R, tminlo, lane);
+                    }
+                }
                 finished = !full && lastT > lmin;                  // rows are sorted: nothing later is <= lmin
             }
             __syncwarp();
             --inflight;
             slot_p = slot_p + 1 == FILTER_STAGES ? 0 : slot_p + 1;
-            if (++cp == req_p) {
-                if (!finished && !full && cp < nchunks) {
+            if (i0 + L == req_p) {
+                if (!finished && !full && req_p < R) {
                     // the request ended before the row did: continue with plain loads
-                    for (int i0 = cp * FILTER_CHUNK; i0 < R; i0 += 64) {
-                        const int i = i0 + 2 * lane;
+                    for (int j0 = req_p; j0 < R; j0 += 64) {
+                        const int i = j0 + 2 * lane;
                         const bool va = i < R, vb = i + 1 < R;
                         const uint32_t Ta = va ? (uint32_t)(uint64_t)ldg64(row_p + i) - tminlo : 0xffffffffu;
                         const uint32_t Tb = vb ? (uint32_t)(uint64_t)ldg64(row_p + i + 1) - tminlo : 0xffffffffu;
@@ -434,6 +466,8 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
                 }
                 cp = 0; ++jp; row_p += rstride; finished = false;
                 req_p = __shfl_sync(FULL, req, min(jp, 31));
+            } else {
+                ++cp;
             }
         }
     }
