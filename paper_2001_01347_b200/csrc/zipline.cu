@@ -85,6 +85,12 @@ struct FilterBufs {
     uint64_t *list2;     // [B][nbk][capb]    survivors of the refinement
     int32_t cells, fcells, nbk, capb, grp;   // grp: fewest buckets per CTA of the bucket sweep
     int32_t nreg, regcap, list1cap;          // set per call: regions per instance and their capacity
+    // SUM bucket route (all nullptr / 0 when the route is off): the timeline is cut into `scells` uniform
+    // cells; runs of cells form buckets of about `sM` elements; `stiles` tiles of TILE_BK buckets each.
+    uint32_t *bnd;                           // [B][stiles*15 + 1]   time at which each bucket starts (non-decreasing)
+    unsigned long long *cellacc;             // [B][scells + 1 + stiles*15 + 1]  scratch of the bucket plan
+    uint16_t *itab;                          // [B][stiles][n][16]   per row: index of its first element in each bucket of the tile
+    int32_t scells, sM, scap, stiles;        // scells == 0: every instance is a single bucket (n * R <= scap)
 };
 
 struct SweepParams {
@@ -999,6 +1005,241 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
     }
 }
 
+// ------------------------------------------------------------------------------ SUM bucket route
+// Every element matters for the prefix sums of the SUM objective, so the whole instance is put into
+// time order - but never as one list in HBM.  The timeline is cut into buckets of about sM elements:
+//   k_sum_plan     per instance: expected element density over uniform time cells from the rows' end points
+//                  (rows are close to arithmetic), cumulated; a bucket is the run of cells whose cumulated
+//                  expectation falls into the same multiple of sM.
+//   k_sum_index    one streaming pass: a warp per row reads the row in storage order and notes, for every
+//                  bucket, the index of the row's first element in it (the index table; 2 bytes per row
+//                  and bucket, tiles of TILE_BK buckets with 16 boundaries each).
+//   k_sum_buckets  a CTA takes the buckets of a tile one after the other: it gathers each row's run
+//                  [start, end) with independent loads (K2: delta from the row neighbour, first flag =
+//                  delta == T), sorts the bucket in shared memory (K1 restricted to the bucket), scans delta
+//                  and flag (K3) with the carry-in that the predecessors of the runs give directly
+//                  (S = sum over rows of the last element before the bucket, cnt = rows that have one),
+//                  evaluates n*T - S where cnt == n (K4) and keeps the first minimum (K5, per tile).
+// A bucket that holds more than scap elements (rows far from arithmetic) sends its instance to the
+// segment sweep instead.
+constexpr int TILE_BK = 15;           // buckets per tile: 16 boundaries = 32 bytes per row and tile
+constexpr int SUM_FP = 12;            // fixed-point bits of the expected counts
+
+// In-place prefix sum of a[0..len) by the whole block; tmp: 34 shared 64-bit words.
+template <bool EXCLUSIVE>
+__device__ void block_prefix_sum_inplace(unsigned long long *a, int len, uint64_t *tmp) {
+    const int tid = threadIdx.x, nt = blockDim.x;
+    const int per = (len + nt - 1) / nt;
+    const int c0 = min(tid * per, len), c1 = min(c0 + per, len);
+    uint64_t loc = 0;
+    for (int c = c0; c < c1; ++c) loc += a[c];
+    uint64_t tot;
+    uint64_t run = block_scan_excl<uint64_t>(loc, OpAdd(), 0ull, tmp, &tot);
+    for (int c = c0; c < c1; ++c) {
+        const uint64_t v = a[c];
+        if (EXCLUSIVE) { a[c] = run; run += v; } else { run += v; a[c] = run; }
+    }
+    __syncthreads();
+}
+
+__global__ void __launch_bounds__(1024) k_sum_plan(const int64_t *ts, int n, int R, InstMeta *meta, FilterBufs F) {
+    grid_dep_wait();
+    __shared__ uint64_t tmp[34];
+    const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+    const InstMeta M = meta[b];
+    if (b == 0 && tid == 0) F.flags[2] = 1;                       // k_finalize writes every instance's outputs
+    if (M.status != ZL_OK) return;
+    if (!M.use32) { if (tid == 0) F.flags[1] = 1; return; }      // wide times: the segment sweep
+    if (F.scells == 0) {                                          // the instance is one bucket
+        if (tid == 0) { meta[b].cscale = 1; meta[b].count = 1; meta[b].count2 = 1; }
+        return;
+    }
+    const uint32_t cells = (uint32_t)F.scells;
+    // (T - 1) < tend for every T, so ((T - 1) * cscale) >> 32 < cells
+    const uint32_t cscale = (uint32_t)max((uint64_t)1, min((uint64_t)0xffffffffu, ((uint64_t)cells << 32) / M.tend));
+    unsigned long long *acc = F.cellacc + (size_t)b * ((size_t)cells + 2 + (size_t)F.stiles * TILE_BK);
+    for (uint32_t c = tid; c <= cells; c += nt) acc[c] = 0;
+    __syncthreads();
+    const int64_t *inst = ts + (size_t)b * n * R;
+    const uint32_t tminlo = (uint32_t)(uint64_t)M.tmin - 1u;
+    // a row spreads its R elements evenly over the cells between its first and its last element
+    for (int p = tid; p < n; p += nt) {
+        const uint32_t e1 = (uint32_t)(uint64_t)ldg64(inst + (size_t)p * R) - tminlo;
+        const uint32_t eR = (uint32_t)(uint64_t)ldg64(inst + (size_t)p * R + R - 1) - tminlo;
+        const uint32_t c1 = cell_of(e1, cscale), cR = cell_of(eR, cscale);
+        const unsigned long long x = ((unsigned long long)R << SUM_FP) / (unsigned long long)(cR - c1 + 1);
+        atomicAdd(&acc[c1], x);
+        atomicAdd(&acc[cR + 1], 0ull - x);
+    }
+    __syncthreads();
+    block_prefix_sum_inplace<false>(acc, (int)cells, tmp);        // expected elements per cell
+    if (tid == 0) acc[cells] = 0;
+    __syncthreads();
+    block_prefix_sum_inplace<true>(acc, (int)cells + 1, tmp);     // expected elements before each cell; [cells]: all
+    // bucket k starts where the cumulated expectation reaches k * sM (linear inside a cell)
+    const unsigned long long per_bucket = (unsigned long long)F.sM << SUM_FP;
+    const uint32_t nbmax = (uint32_t)(F.stiles * TILE_BK);
+    const uint32_t nbk = (uint32_t)max(1ull, min((unsigned long long)nbmax, (acc[cells] + per_bucket - 1) / per_bucket));
+    unsigned long long *bnd64 = acc + cells + 1;                  // scratch: nbk + 1 words behind the cells
+    for (uint32_t c = tid; c < cells; c += nt) {
+        const unsigned long long lo = acc[c], hi = acc[c + 1];
+        if (hi == lo) continue;
+        const unsigned long long start = ((unsigned long long)c << 32) / cscale + 1, next = ((unsigned long long)(c + 1) << 32) / cscale + 1;
+        for (unsigned long long k = max(1ull, (lo + per_bucket - 1) / per_bucket); k < nbk && k * per_bucket < hi; ++k)
+            bnd64[k] = start + (k * per_bucket - lo) * (next - start) / (hi - lo);
+    }
+    if (tid == 0) { bnd64[0] = 0; bnd64[nbk] = 0xffffffffull; }
+    __syncthreads();
+    {   // boundaries must not decrease: inclusive prefix maximum
+        const int len = (int)nbk + 1, per = (len + nt - 1) / nt;
+        const int k0 = min(tid * per, len), k1 = min(k0 + per, len);
+        uint64_t loc = 0;
+        for (int k = k0; k < k1; ++k) loc = max(loc, (uint64_t)bnd64[k]);
+        uint64_t tot;
+        uint64_t run = block_scan_excl<uint64_t>(loc, OpMax(), 0ull, tmp, &tot);
+        uint32_t *bnd = F.bnd + (size_t)b * (nbmax + 1);
+        for (int k = k0; k < k1; ++k) { run = max(run, (uint64_t)bnd64[k]); bnd[k] = (uint32_t)min(run, (uint64_t)0xffffffffu); }
+    }
+    if (tid == 0) {
+        meta[b].cscale = cscale;
+        meta[b].count = nbk;                                      // buckets of this instance
+        meta[b].count2 = (nbk + TILE_BK - 1) / TILE_BK;           // tiles
+    }
+}
+
+// Boundary k of a row (k = 0..buckets) is the index of its first element in a bucket >= k.  Tile t keeps
+// boundaries 15t .. 15t + 15, so a multiple of 15 is stored twice (last slot of one tile, first of the next).
+__device__ __forceinline__ void index_entry(uint16_t *tab, int n, int stiles, int row, int k, int i) {
+    const int t = k / TILE_BK, s = k - t * TILE_BK;
+    if (t < stiles) tab[((size_t)t * n + row) * 16 + s] = (uint16_t)i;
+    if (s == 0 && t > 0) tab[((size_t)(t - 1) * n + row) * 16 + TILE_BK] = (uint16_t)i;
+}
+
+constexpr int INDEX_UNROLL = 4;       // 32-element steps loaded before any is used
+
+// Largest k in [lo, hi] with a[k] <= T, given a[lo] <= T.
+__device__ __forceinline__ int bucket_search(const uint32_t *a, int lo, int hi, uint32_t T) {
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (a[mid] <= T) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+__global__ void __launch_bounds__(256) k_sum_index(const int64_t *ts, int n, int R, const InstMeta *meta, FilterBufs F) {
+    grid_dep_wait();
+    extern __shared__ __align__(16) unsigned char smem[];
+    uint32_t *a = (uint32_t *)smem;                               // bucket start times, [nbk + 1]
+    const int b = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const InstMeta M = meta[b];
+    if (M.status != ZL_OK || M.cscale == 0) return;
+    const uint32_t tminlo = (uint32_t)(uint64_t)M.tmin - 1u;
+    const int nbk = (int)M.count;
+    const uint32_t *bg = F.bnd + (size_t)b * (F.stiles * TILE_BK + 1);
+    for (int k = threadIdx.x; k <= nbk; k += blockDim.x) a[k] = bg[k];
+    __syncthreads();
+    uint16_t *tab = F.itab + (size_t)b * F.stiles * n * 16;
+    for (int row = blockIdx.x * nw + warp; row < n; row += gridDim.x * nw) {
+        const int64_t *rp = ts + ((size_t)b * n + row) * R;
+        int carry = -1;                                           // bucket of the element before this step (-1: none)
+        int kc = 0;                                               // the same, as the lower end of the next search
+        // position R counts as an element of bucket `nbk`: it closes every bucket after the row's last one
+        for (int i0 = 0; i0 <= R; i0 += 32 * INDEX_UNROLL) {
+            int64_t v[INDEX_UNROLL];
+#pragma unroll
+            for (int u = 0; u < INDEX_UNROLL; ++u) {
+                const int i = i0 + 32 * u + lane;
+                v[u] = i < R ? ldg64(rp + i) : 0;
+            }
+#pragma unroll
+            for (int u = 0; u < INDEX_UNROLL; ++u) {
+                const int ibase = i0 + 32 * u, i = ibase + lane;
+                int k = nbk;
+                if (ibase < R) {                                  // warp-uniform: the step holds elements of the row
+                    const uint32_t T = (uint32_t)(uint64_t)v[u] - tminlo;
+                    const uint32_t Tlast = __shfl_sync(FULL, T, min(31, R - 1 - ibase));
+                    const int khi = bucket_search(a, kc, nbk - 1, Tlast);    // the same search in every lane
+                    if (i < R) k = bucket_search(a, kc, khi, T);
+                    kc = khi;
+                }
+                int kp = __shfl_up_sync(FULL, k, 1);
+                if (lane == 0) kp = carry;
+                carry = __shfl_sync(FULL, k, 31);
+                if (i <= R)
+                    for (int kk = kp + 1; kk <= k; ++kk) index_entry(tab, n, F.stiles, row, kk, i);
+            }
+        }
+    }
+}
+
+__global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, int R, int B, int G, InstMeta *meta, FilterBufs F,
+                                                     int nres, SegResult *seg) {
+    grid_dep_wait();
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ uint64_t tmp[34];
+    __shared__ unsigned int sstatus;
+    __shared__ InstMeta sM;
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+    const int NG = nt / G, gi = tid / G, g = tid % G;
+    const int cap = F.scap;
+    Key<uint32_t> *keys = (Key<uint32_t> *)smem;
+    const BatchWS<uint32_t> ws{keys, keys + cap, (uint32_t *)(keys + 2 * (size_t)cap), cap};
+    const bool single = F.scells == 0;
+    for (int item = blockIdx.x; item < F.stiles * B; item += gridDim.x) {
+        const int b = item / F.stiles, t = item - b * F.stiles;
+        __syncthreads();                                          // shared state of the previous item is done with
+        if (tid == 0) { sM = meta[b]; sstatus = 0; }              // one read: another CTA may set `overflow` meanwhile
+        __syncthreads();
+        const InstMeta M = sM;
+        if (M.status != ZL_OK || M.cscale == 0 || M.overflow || t >= (int)M.count2) continue;
+        const int64_t *inst = ts + (size_t)b * n * R;
+        const uint32_t tminlo = (uint32_t)(uint64_t)M.tmin - 1u;
+        const uint16_t *tab = single ? nullptr : F.itab + ((size_t)b * F.stiles + t) * n * 16;
+        const int j1 = min(TILE_BK, (int)M.count - t * TILE_BK);  // buckets of this tile
+        uint64_t bd = ~0ull, bt = ~0ull;
+        bool over = false;
+        for (int j = 0; j < j1 && !over; ++j) {
+            // runs [s, e) of this group's rows: element count, and the carry-in from the runs' predecessors
+            uint32_t mycnt = 0, myC = 0;
+            uint64_t myS = 0;
+            if (g == 0) {
+                for (int r = gi; r < n; r += NG) {
+                    const int s = single ? 0 : (int)__ldg(tab + (size_t)r * 16 + j);
+                    const int e = single ? R : (int)__ldg(tab + (size_t)r * 16 + j + 1);
+                    mycnt += (uint32_t)(e - s);
+                    if (s > 0) { myS += (uint32_t)(uint64_t)ldg64(inst + (size_t)r * R + s - 1) - tminlo; ++myC; }
+                }
+            }
+            uint64_t totcc, totS;
+            const uint64_t offcc = block_scan_excl<uint64_t>(((uint64_t)myC << 32) | mycnt, OpAdd(), 0ull, tmp, &totcc);
+            block_scan_excl<uint64_t>(myS, OpAdd(), 0ull, tmp, &totS);
+            const uint32_t m = (uint32_t)totcc;
+            if (m > (uint32_t)cap) { over = true; break; }
+            uint32_t o = (uint32_t)__shfl_sync(FULL, (uint32_t)offcc, lane - g);
+            for (int r = gi; r < n; r += NG) {
+                const int s = single ? 0 : (int)__ldg(tab + (size_t)r * 16 + j);
+                const int e = single ? R : (int)__ldg(tab + (size_t)r * 16 + j + 1);
+                const int64_t *rp = inst + (size_t)r * R;
+                for (int i = s + g; i < e; i += G) {
+                    const uint32_t T = (uint32_t)(uint64_t)ldg64(rp + i) - tminlo;
+                    const uint32_t pv = i > 0 ? (uint32_t)(uint64_t)ldg64(rp + i - 1) - tminlo : 0u;
+                    keys[o + (uint32_t)(i - s)] = Key<uint32_t>::make(T, T - pv);
+                }
+                o += (uint32_t)(e - s);
+            }
+            __syncthreads();
+            uint64_t cS = totS;
+            uint32_t cC = (uint32_t)(totcc >> 32);
+            run_batch<uint32_t, ZL_OBJ_SUM>(ws, (int)m, (uint32_t)M.t0, n, tmp, (uint32_t)0, cS, cC, bd, bt);
+        }
+        if (over) {                                               // uniform over the block
+            if (tid == 0) { meta[b].overflow = 1; F.flags[1] = 1; }
+            continue;
+        }
+        block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres + t]);
+    }
+}
+
 // Index of the last element of a sorted row that is <= bar (-1 if none).  Rows are close to arithmetic, so the
 // position is first guessed from the row's end points, bracketed by doubling steps around the guess, then bisected.
 __device__ int last_index_not_after(const int64_t *row, int R, int64_t bar) {
@@ -1122,7 +1363,7 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
     const int b = blockIdx.y, tid = threadIdx.x;
     if (filter && F.flags[2] == 0) return;                        // k_tail finished every instance of this call
     const InstMeta M = meta[b];
-    if (M.status == ZL_OK && handled_by_filter(M, filter) && tail_instance(M)) return;   // finished by k_tail
+    if (objective == ZL_OBJ_RANGE && M.status == ZL_OK && handled_by_filter(M, filter) && tail_instance(M)) return;   // finished by k_tail
     __shared__ uint64_t red[34];
     __shared__ unsigned int sstatus;
     __shared__ SegResult best;
@@ -1131,7 +1372,9 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
     uint64_t bd = ~0ull, bt = ~0ull;
     uint32_t st = M.status;
     if (st == ZL_OK) {
-        const int used = !handled_by_filter(M, filter) ? nseg : tail_instance(M) ? 1 : (F.nbk + bucket_group(F, M.count2) - 1) / bucket_group(F, M.count2);
+        const int used = !handled_by_filter(M, filter) ? nseg
+                         : objective == ZL_OBJ_SUM ? (int)M.count2                      // bucket route: one result per tile
+                         : tail_instance(M) ? 1 : (F.nbk + bucket_group(F, M.count2) - 1) / bucket_group(F, M.count2);
         for (int s = tid; s < used; s += blockDim.x) {
             const SegResult r = seg[(size_t)b * nres + s];
             if (r.status != ZL_OK) st = max(st, (uint32_t)r.status);
@@ -1419,8 +1662,9 @@ void launch_dep(bool early, void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
 
 void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_t *ev) {
     const bool filter = q.fb.table != nullptr && q.objective == ZL_OBJ_RANGE;
+    const bool sumfast = q.fb.flags != nullptr && q.fb.scap != 0 && q.objective == ZL_OBJ_SUM;
     zl::FilterBufs fb = q.fb;
-    if (!filter) memset(&fb, 0, sizeof(fb));
+    if (!filter && !sumfast) memset(&fb, 0, sizeof(fb));
     if (ev) cudaEventRecord(ev[0], st);
     // many small instances: small CTAs so that several share an SM; few large ones: one large CTA each
     const bool many = q.B > 2 * q.num_sms;
@@ -1458,23 +1702,42 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         const int bthreads = std::max(64, std::min(256, fb.capb / 4));
         launch_dep(!((q.pdl_off >> 6) & 1), zl::k_buckets, dim3(std::min(ngroups * q.B, wide)), dim3(bthreads), (size_t)fb.capb * 20, st,
                    (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg, q.B);
+    } else if (sumfast) {
+        const bool single = fb.scells == 0;
+        launch_dep(!((q.pdl_off >> 1) & 1), zl::k_sum_plan, dim3(q.B), dim3(single ? 32 : 1024), 0, st, q.ts, q.n, q.R, q.meta, fb);
+        if (!single) {
+            const int nw = 8;
+            const int row_blocks = std::max(1, std::min((q.n + nw - 1) / nw, (32 * q.num_sms + q.B - 1) / q.B));
+            launch_dep(!((q.pdl_off >> 2) & 1), zl::k_sum_index, dim3(row_blocks, q.B), dim3(32 * nw), ((size_t)fb.stiles * zl::TILE_BK + 1) * 4, st, q.ts, q.n, q.R,
+                       (const zl::InstMeta *)q.meta, fb);
+        }
+        if (ev) cudaEventRecord(ev[2], st);
+        const long long N = (long long)q.n * q.R;
+        int bthreads = single ? (int)std::max<long long>(64, std::min<long long>(1024, pow2_ceil((int)((N + 3) / 4))))
+                              : (fb.scap > 4096 ? 1024 : 512);
+        if (q.tail_threads) bthreads = q.tail_threads;
+        const int G = std::max(1, std::min(32, pow2_floor(std::max(1, bthreads / q.n))));
+        const int items = fb.stiles * q.B;
+        launch_dep(!((q.pdl_off >> 3) & 1), zl::k_sum_buckets, dim3(std::min(items, 32 * q.num_sms)), dim3(bthreads), (size_t)fb.scap * 20, st,
+                   q.ts, q.n, q.R, q.B, G, q.meta, fb, q.nres, q.seg);
     } else if (ev) {
         cudaEventRecord(ev[2], st);
     }
     zl::SweepParams sp;
     sp.ts = q.ts; sp.meta = q.meta; sp.seg = q.seg;
     sp.n = q.n; sp.R = q.R; sp.B = q.B; sp.nseg = p.nseg; sp.nres = q.nres; sp.G = p.G; sp.cap = p.cap;
-    sp.flags = q.flags; sp.target = p.target; sp.filter = filter ? 1 : 0;
-    sp.need = filter ? fb.flags : nullptr;
-    // with the filter route on, the segment sweep is only the fallback: a small persistent grid
+    const bool fast = filter || sumfast;
+    sp.flags = q.flags; sp.target = p.target; sp.filter = fast ? 1 : 0;
+    sp.need = fast ? fb.flags : nullptr;
+    // with a fast route on, the segment sweep is only the fallback: a small persistent grid
     const int items = p.nseg * q.B;
-    const int sweep_ctas = filter ? std::min(items, 2 * q.num_sms) : items;
+    const int sweep_ctas = fast ? std::min(items, 2 * q.num_sms) : items;
     if (q.objective == ZL_OBJ_RANGE) launch_dep(!((q.pdl_off >> 7) & 1), zl::k_sweep<ZL_OBJ_RANGE>, dim3(sweep_ctas), dim3(p.threads), p.smem, st, sp);
     else launch_dep(!((q.pdl_off >> 7) & 1), zl::k_sweep<ZL_OBJ_SUM>, dim3(sweep_ctas), dim3(p.threads), p.smem, st, sp);
     if (ev) cudaEventRecord(ev[3], st);
     const int fthreads = std::max(32, std::min(256, pow2_ceil(q.n)));
     launch_dep(!((q.pdl_off >> 8) & 1), zl::k_finalize, dim3((q.n + fthreads - 1) / fthreads, q.B), dim3(fthreads), 0, st, q.ts, q.n, q.R, p.nseg, fb, q.nres, q.objective,
-                                                                  filter ? 1 : 0, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
+                                                                  fast ? 1 : 0, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
     if (ev) cudaEventRecord(ev[4], st);
 }
 
@@ -1484,6 +1747,7 @@ cudaError_t raise_shared_memory_limits() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_buckets, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_tail, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_buckets, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     return e;
 }
 
@@ -1586,6 +1850,35 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
             filter_b += sizes[i];
         }
     }
+    if (cfg->objective == ZL_OBJ_SUM) {
+        // bucket route: shared-memory batches of scap elements, buckets of about 11/16 of that
+        const long long N = (long long)cfg->n_workers * cfg->lookahead_R;
+        const size_t mb = (size_t)cfg->max_batch;
+        zl::FilterBufs &f = h->fb;
+        f.scap = N <= 4096 ? std::max(64, pow2_ceil((int)N)) : cfg->n_workers > 2048 ? 8192 : 4096;
+        f.stiles = 1;
+        bool on = true;
+        if (N > f.scap) {
+            f.sM = f.scap / 16 * 11;
+            const long long nbk = N / f.sM + 1;
+            f.stiles = (int)((nbk + zl::TILE_BK - 1) / zl::TILE_BK);
+            f.scells = (int)std::max<long long>(1024, std::min<long long>(1 << 16, pow2_ceil((int)std::min<long long>(N / 64, 1 << 20))));
+            on = nbk <= 12000 && cfg->lookahead_R <= 65535;       // boundaries fit shared memory, row indices are 16-bit
+        }
+        if (on) {
+            const size_t nb1 = (size_t)f.stiles * zl::TILE_BK + 1;
+            const size_t sizes[4] = {mb * nb1 * 4, mb * ((size_t)f.scells + 1 + nb1) * 8,
+                                     f.scells ? mb * f.stiles * cfg->n_workers * 32 : 64, 64};
+            void **ptrs[4] = {(void **)&f.bnd, (void **)&f.cellacc, (void **)&f.itab, (void **)&f.flags};
+            for (int i = 0; i < 4; ++i) {
+                if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
+                filter_b += sizes[i];
+            }
+            h->nres = std::max(zl::MAX_SEGMENTS, f.stiles);
+        } else {
+            memset(&f, 0, sizeof(f));
+        }
+    }
     const size_t seg_b = (size_t)cfg->max_batch * h->nres * sizeof(zl::SegResult);
     if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_meta, meta_b);
     if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_seg, seg_b);
@@ -1597,6 +1890,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
         cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
         cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
+        cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab);
         delete h;
         return st;
     }
@@ -1659,6 +1953,7 @@ zl_status zl_destroy(zl_handle *h) {
     cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
     cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
     cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
+    cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab);
     cudaFree(h->s_ts); cudaFree(h->s_idx); cudaFree(h->s_barrier); cudaFree(h->s_wait); cudaFree(h->s_status);
     if (h->s_stream) cudaStreamDestroy(h->s_stream);
     zl_profile_end(h);
@@ -1704,7 +1999,8 @@ size_t zl_workspace_bytes(const zl_handle *h) { return h ? h->ws_bytes + h->stag
 int32_t zl_launches_per_call(const zl_handle *h) {
     if (!h) return 0;
     const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter;
-    return 3 + (filter ? 6 : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
+    const bool sumfast = h->cfg.objective == ZL_OBJ_SUM && !h->opt_no_filter && h->fb.scap != 0;
+    return 3 + (filter ? 6 : 0) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
 }
 int32_t zl_segments_per_instance(const zl_handle *h, int32_t B) { return h && B >= 1 ? make_plan(h, B).nseg : 0; }
 int32_t zl_last_cuda_error(const zl_handle *h) { return h ? h->last_cuda_error : 0; }
@@ -1728,7 +2024,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.fb = h->fb;
     q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.pdl_off = h->opt_pdl_off;
     q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
-    if (h->opt_no_filter) q.fb.table = nullptr;
+    if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, st, ev);
     if (ev) ++h->prof_calls;

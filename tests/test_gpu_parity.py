@@ -25,14 +25,15 @@ def gpu_select(ts_np, objective, flags=0, options=None):
     sel = h.select_batched(d_ts)
     torch.cuda.synchronize()
     got = (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy())
-    if objective == 0 and "no_filter" not in (options or {}):
-        # RANGE has two routes (filter pass + one sort, or the segment sweep): both must agree exactly
+    if "no_filter" not in (options or {}):
+        # each objective has two routes (RANGE: filter pass + one sort, SUM: time buckets; or the segment
+        # sweep for both): they must agree exactly
         h.set_option("no_filter", 1)
         sel2 = h.select_batched(d_ts)
         torch.cuda.synchronize()
         for a, b in zip(got, (sel2.idx.cpu().numpy(), sel2.barrier.cpu().numpy(), sel2.wait.cpu().numpy(),
                               sel2.status.cpu().numpy())):
-            assert (a == b).all(), "filter route and segment-sweep route disagree"
+            assert (a == b).all(), "fast route and segment-sweep route disagree"
     h.destroy()
     return got
 
@@ -272,6 +273,55 @@ def test_mixed_batch_of_routes():
     sel, filtered, refined, overflow = _routes(ts)
     assert overflow.tolist() == [0, 0, 1, 0, 0]
     assert_same(ts, 0, (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()))
+
+
+# ---------------------------------------------------------------- the SUM routes
+def _sum_routes(ts_np):
+    B, n, R = ts_np.shape
+    h = zl.ZipLine(n, R, B, 1)
+    sel = h.select_batched(torch.from_numpy(ts_np).cuda())
+    torch.cuda.synchronize()
+    buckets, tiles, overflow = h.filter_counts(B)
+    h.destroy()
+    got = (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy())
+    return got, np.array(buckets), np.array(tiles), np.array(overflow)
+
+
+def test_sum_routes_are_all_exercised_and_exact():
+    # one bucket: the whole instance fits a shared-memory batch
+    ts = zi.generate(zi.CONFIGS["c2"].with_(B=5, n=24, R=100))
+    got, buckets, tiles, overflow = _sum_routes(ts)
+    assert (buckets == 1).all() and (tiles == 1).all() and (overflow == 0).all()
+    assert_same(ts, 1, got)
+    # several tiles of buckets, ragged last tile, rows of very different speeds
+    ts = zi.generate(zi.CONFIGS["c4"].with_(B=3, n=200, R=700))
+    got, buckets, tiles, overflow = _sum_routes(ts)
+    assert (buckets > 30).all() and (tiles >= 3).all() and (overflow == 0).all()
+    assert_same(ts, 1, got)
+    # start offsets and two speeds (the rows do not start together)
+    ts = zi.generate(zi.CONFIGS["c5"].with_(B=2, n=300, R=500))
+    got, buckets, tiles, overflow = _sum_routes(ts)
+    assert (buckets > 15).all() and (overflow == 0).all()
+    assert_same(ts, 1, got)
+    # rows far from arithmetic (quadratic growth): the early buckets overflow, the segment sweep takes over
+    row = np.cumsum(np.arange(1, 401)) * 1000
+    ts = np.broadcast_to(row, (2, 200, 400)).astype(np.int64).copy()
+    ts += np.arange(200)[None, :, None]
+    got, buckets, tiles, overflow = _sum_routes(ts)
+    assert (overflow == 1).all()
+    assert_same(ts, 1, got)
+
+
+def test_sum_mixed_batch_of_routes():
+    # a regular, an overflowing and a wide-span instance in one batch
+    n, R = 128, 512
+    regular = zi.generate(zi.CONFIGS["c4"].with_(B=1, n=n, R=R))[0]
+    quad = (np.cumsum(np.arange(1, R + 1)) * 2000)[None, :] + np.arange(n)[:, None]
+    wide = regular * 50_000
+    ts = np.stack([regular, quad, wide, regular + 5]).astype(np.int64)
+    got, buckets, tiles, overflow = _sum_routes(ts)
+    assert overflow.tolist() == [0, 1, 0, 0] and buckets[2] == 0
+    assert_same(ts, 1, got)
 
 
 # ---------------------------------------------------------------- extreme shapes
