@@ -1009,8 +1009,8 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
 // Every element matters for the prefix sums of the SUM objective, so the whole instance is put into
 // time order - but never as one list in HBM.  The timeline is cut into buckets of about sM elements:
 //   k_sum_plan     per instance: expected element density over uniform time cells from the rows' end points
-//                  (rows are close to arithmetic), cumulated; a bucket is the run of cells whose cumulated
-//                  expectation falls into the same multiple of sM.
+//                  (rows are close to arithmetic), cumulated; bucket k starts at the time where the cumulated
+//                  expectation reaches k * sM.
 //   k_sum_index    one streaming pass: a warp per row reads the row in storage order and notes, for every
 //                  bucket, the index of the row's first element in it (the index table; 2 bytes per row
 //                  and bucket, tiles of TILE_BK buckets with 16 boundaries each).
@@ -1025,25 +1025,41 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
 constexpr int TILE_BK = 15;           // buckets per tile: 16 boundaries = 32 bytes per row and tile
 constexpr int SUM_FP = 12;            // fixed-point bits of the expected counts
 
-// In-place prefix sum of a[0..len) by the whole block; tmp: 34 shared 64-bit words.
-template <bool EXCLUSIVE>
-__device__ void block_prefix_sum_inplace(unsigned long long *a, int len, uint64_t *tmp) {
-    const int tid = threadIdx.x, nt = blockDim.x;
-    const int per = (len + nt - 1) / nt;
-    const int c0 = min(tid * per, len), c1 = min(c0 + per, len);
-    uint64_t loc = 0;
-    for (int c = c0; c < c1; ++c) loc += a[c];
-    uint64_t tot;
-    uint64_t run = block_scan_excl<uint64_t>(loc, OpAdd(), 0ull, tmp, &tot);
-    for (int c = c0; c < c1; ++c) {
-        const uint64_t v = a[c];
-        if (EXCLUSIVE) { a[c] = run; run += v; } else { run += v; a[c] = run; }
+// In-place prefix scan of a shared-memory array by the whole block: every warp takes a contiguous piece
+// and walks it 32 elements a step.  tmp: 32 shared words of T.  Every thread calls.
+template <typename T, typename Op, bool EXCLUSIVE>
+__device__ void smem_scan_inplace(T *a, int len, Op op, T identity, T *tmp) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const int seg = (((len + nw - 1) / nw) + 31) & ~31;
+    const int w0 = min(warp * seg, len), w1 = min(w0 + seg, len);
+    T tot = identity;
+    for (int i = w0 + lane; i < w1; i += 32) tot = op(tot, a[i]);
+    tot = warp_reduce(tot, op);
+    if (lane == 0) tmp[warp] = tot;
+    __syncthreads();
+    T carry = identity;
+    for (int w = 0; w < warp; ++w) carry = op(carry, tmp[w]);
+    for (int base = w0; base < w1; base += 32) {
+        const int i = base + lane;
+        const T v = i < w1 ? a[i] : identity;
+        T inc = v;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const T y = shfl_up(inc, d);
+            if (lane >= d) inc = op(y, inc);
+        }
+        T exc = shfl_up(inc, 1);
+        if (lane == 0) exc = identity;
+        if (i < w1) a[i] = op(carry, EXCLUSIVE ? exc : inc);
+        carry = op(carry, shfl_idx(inc, 31));
     }
     __syncthreads();
 }
 
+// Dynamic shared memory: (scells + 1) 64-bit cell accumulators, then stiles * TILE_BK + 1 32-bit boundaries.
 __global__ void __launch_bounds__(1024) k_sum_plan(const int64_t *ts, int n, int R, InstMeta *meta, FilterBufs F) {
     grid_dep_wait();
+    extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
     const InstMeta M = meta[b];
@@ -1055,9 +1071,10 @@ __global__ void __launch_bounds__(1024) k_sum_plan(const int64_t *ts, int n, int
         return;
     }
     const uint32_t cells = (uint32_t)F.scells;
+    unsigned long long *acc = (unsigned long long *)smem;
+    uint32_t *bsm = (uint32_t *)(acc + cells + 1);
     // (T - 1) < tend for every T, so ((T - 1) * cscale) >> 32 < cells
     const uint32_t cscale = (uint32_t)max((uint64_t)1, min((uint64_t)0xffffffffu, ((uint64_t)cells << 32) / M.tend));
-    unsigned long long *acc = F.cellacc + (size_t)b * ((size_t)cells + 2 + (size_t)F.stiles * TILE_BK);
     for (uint32_t c = tid; c <= cells; c += nt) acc[c] = 0;
     __syncthreads();
     const int64_t *inst = ts + (size_t)b * n * R;
@@ -1072,34 +1089,28 @@ __global__ void __launch_bounds__(1024) k_sum_plan(const int64_t *ts, int n, int
         atomicAdd(&acc[cR + 1], 0ull - x);
     }
     __syncthreads();
-    block_prefix_sum_inplace<false>(acc, (int)cells, tmp);        // expected elements per cell
+    smem_scan_inplace<unsigned long long, OpAdd, false>(acc, (int)cells, OpAdd(), 0ull, (unsigned long long *)tmp);   // expected elements per cell
     if (tid == 0) acc[cells] = 0;
     __syncthreads();
-    block_prefix_sum_inplace<true>(acc, (int)cells + 1, tmp);     // expected elements before each cell; [cells]: all
+    smem_scan_inplace<unsigned long long, OpAdd, true>(acc, (int)cells + 1, OpAdd(), 0ull, (unsigned long long *)tmp);  // ... before each cell; [cells]: all
     // bucket k starts where the cumulated expectation reaches k * sM (linear inside a cell)
     const unsigned long long per_bucket = (unsigned long long)F.sM << SUM_FP;
     const uint32_t nbmax = (uint32_t)(F.stiles * TILE_BK);
     const uint32_t nbk = (uint32_t)max(1ull, min((unsigned long long)nbmax, (acc[cells] + per_bucket - 1) / per_bucket));
-    unsigned long long *bnd64 = acc + cells + 1;                  // scratch: nbk + 1 words behind the cells
     for (uint32_t c = tid; c < cells; c += nt) {
         const unsigned long long lo = acc[c], hi = acc[c + 1];
         if (hi == lo) continue;
+        unsigned long long k = max(1ull, (lo + per_bucket - 1) / per_bucket);
+        if (k >= nbk || k * per_bucket >= hi) continue;
         const unsigned long long start = ((unsigned long long)c << 32) / cscale + 1, next = ((unsigned long long)(c + 1) << 32) / cscale + 1;
-        for (unsigned long long k = max(1ull, (lo + per_bucket - 1) / per_bucket); k < nbk && k * per_bucket < hi; ++k)
-            bnd64[k] = start + (k * per_bucket - lo) * (next - start) / (hi - lo);
+        for (; k < nbk && k * per_bucket < hi; ++k)
+            bsm[k] = (uint32_t)min(0xfffffffeull, start + (k * per_bucket - lo) * (next - start) / (hi - lo));
     }
-    if (tid == 0) { bnd64[0] = 0; bnd64[nbk] = 0xffffffffull; }
+    if (tid == 0) { bsm[0] = 0; bsm[nbk] = 0xffffffffu; }
     __syncthreads();
-    {   // boundaries must not decrease: inclusive prefix maximum
-        const int len = (int)nbk + 1, per = (len + nt - 1) / nt;
-        const int k0 = min(tid * per, len), k1 = min(k0 + per, len);
-        uint64_t loc = 0;
-        for (int k = k0; k < k1; ++k) loc = max(loc, (uint64_t)bnd64[k]);
-        uint64_t tot;
-        uint64_t run = block_scan_excl<uint64_t>(loc, OpMax(), 0ull, tmp, &tot);
-        uint32_t *bnd = F.bnd + (size_t)b * (nbmax + 1);
-        for (int k = k0; k < k1; ++k) { run = max(run, (uint64_t)bnd64[k]); bnd[k] = (uint32_t)min(run, (uint64_t)0xffffffffu); }
-    }
+    smem_scan_inplace<uint32_t, OpMax, false>(bsm, (int)nbk + 1, OpMax(), 0u, (uint32_t *)tmp);   // boundaries must not decrease
+    uint32_t *bnd = F.bnd + (size_t)b * (nbmax + 1);
+    for (uint32_t k = tid; k <= nbk; k += nt) bnd[k] = bsm[k];
     if (tid == 0) {
         meta[b].cscale = cscale;
         meta[b].count = nbk;                                      // buckets of this instance
@@ -1107,8 +1118,9 @@ __global__ void __launch_bounds__(1024) k_sum_plan(const int64_t *ts, int n, int
     }
 }
 
-// Boundary k of a row (k = 0..buckets) is the index of its first element in a bucket >= k.  Tile t keeps
-// boundaries 15t .. 15t + 15, so a multiple of 15 is stored twice (last slot of one tile, first of the next).
+// Boundary k of a row (k = 0..buckets) is the index of its first element at or after the start time of
+// bucket k.  Tile t keeps boundaries 15t .. 15t + 15, so a multiple of 15 is stored twice (last slot of one
+// tile, first of the next).
 __device__ __forceinline__ void index_entry(uint16_t *tab, int n, int stiles, int row, int k, int i) {
     const int t = k / TILE_BK, s = k - t * TILE_BK;
     if (t < stiles) tab[((size_t)t * n + row) * 16 + s] = (uint16_t)i;
@@ -1117,19 +1129,11 @@ __device__ __forceinline__ void index_entry(uint16_t *tab, int n, int stiles, in
 
 constexpr int INDEX_UNROLL = 4;       // 32-element steps loaded before any is used
 
-// Largest k in [lo, hi] with a[k] <= T, given a[lo] <= T.
-__device__ __forceinline__ int bucket_search(const uint32_t *a, int lo, int hi, uint32_t T) {
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (a[mid] <= T) lo = mid; else hi = mid - 1;
-    }
-    return lo;
-}
-
+// Dynamic shared memory: the bucket start times of the instance.
 __global__ void __launch_bounds__(256) k_sum_index(const int64_t *ts, int n, int R, const InstMeta *meta, FilterBufs F) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
-    uint32_t *a = (uint32_t *)smem;                               // bucket start times, [nbk + 1]
+    uint32_t *a = (uint32_t *)smem;                               // [nbk + 1], a[nbk] = 0xffffffff
     const int b = blockIdx.y, lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
     const InstMeta M = meta[b];
     if (M.status != ZL_OK || M.cscale == 0) return;
@@ -1141,10 +1145,8 @@ __global__ void __launch_bounds__(256) k_sum_index(const int64_t *ts, int n, int
     uint16_t *tab = F.itab + (size_t)b * F.stiles * n * 16;
     for (int row = blockIdx.x * nw + warp; row < n; row += gridDim.x * nw) {
         const int64_t *rp = ts + ((size_t)b * n + row) * R;
-        int carry = -1;                                           // bucket of the element before this step (-1: none)
-        int kc = 0;                                               // the same, as the lower end of the next search
-        // position R counts as an element of bucket `nbk`: it closes every bucket after the row's last one
-        for (int i0 = 0; i0 <= R; i0 += 32 * INDEX_UNROLL) {
+        int kc = -1;                                              // boundaries 0..kc of this row are written
+        for (int i0 = 0; i0 < R; i0 += 32 * INDEX_UNROLL) {
             int64_t v[INDEX_UNROLL];
 #pragma unroll
             for (int u = 0; u < INDEX_UNROLL; ++u) {
@@ -1153,38 +1155,101 @@ __global__ void __launch_bounds__(256) k_sum_index(const int64_t *ts, int n, int
             }
 #pragma unroll
             for (int u = 0; u < INDEX_UNROLL; ++u) {
-                const int ibase = i0 + 32 * u, i = ibase + lane;
-                int k = nbk;
-                if (ibase < R) {                                  // warp-uniform: the step holds elements of the row
-                    const uint32_t T = (uint32_t)(uint64_t)v[u] - tminlo;
-                    const uint32_t Tlast = __shfl_sync(FULL, T, min(31, R - 1 - ibase));
-                    const int khi = bucket_search(a, kc, nbk - 1, Tlast);    // the same search in every lane
-                    if (i < R) k = bucket_search(a, kc, khi, T);
-                    kc = khi;
+                const int ibase = i0 + 32 * u;
+                if (ibase >= R) break;                            // warp-uniform
+                // the step's 32 elements, ascending over the lanes; lanes past the row's end hold +inf
+                const uint32_t T = ibase + lane < R ? (uint32_t)(uint64_t)v[u] - tminlo : 0xffffffffu;
+                const uint32_t Tlast = __shfl_sync(FULL, T, min(31, R - 1 - ibase));
+                // every boundary whose bucket starts at or before the step's last element is settled here:
+                // lane l owns boundary kc + 1 + l and counts the elements before its start time
+                for (;;) {
+                    const int kk = kc + 1 + lane;
+                    const uint32_t av = kk <= nbk ? a[kk] : 0xffffffffu;
+                    const bool mine = av <= Tlast;                // a prefix of the lanes: start times do not decrease
+                    int pos = 0;
+#pragma unroll
+                    for (int step = 16; step > 0; step >>= 1) {
+                        const uint32_t tm = __shfl_sync(FULL, T, pos + step - 1);
+                        if (tm < av) pos += step;
+                    }
+                    if (mine) index_entry(tab, n, F.stiles, row, kk, ibase + pos);
+                    const int done = __popc(__ballot_sync(FULL, mine));
+                    kc += done;
+                    if (done < 32) break;
                 }
-                int kp = __shfl_up_sync(FULL, k, 1);
-                if (lane == 0) kp = carry;
-                carry = __shfl_sync(FULL, k, 31);
-                if (i <= R)
-                    for (int kk = kp + 1; kk <= k; ++kk) index_entry(tab, n, F.stiles, row, kk, i);
             }
         }
+        // buckets that start after the row's last element
+        for (int kk = kc + 1 + lane; kk <= nbk; kk += 32) index_entry(tab, n, F.stiles, row, kk, R);
     }
 }
 
-__global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, int R, int B, int G, InstMeta *meta, FilterBufs F,
+// Exclusive prefix sums of two values per thread over the block, in thread order, and both totals.
+// tmp: 68 shared 64-bit words that no call since the block's last two barriers used (callers alternate two
+// buffers, so the call ends without a barrier).  Every thread calls.
+__device__ __forceinline__ void block_scan_add2(uint64_t x1, uint64_t x2, uint64_t &e1, uint64_t &e2, uint64_t &t1,
+                                                uint64_t &t2, uint64_t *tmp) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    uint64_t i1 = x1, i2 = x2;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint64_t y1 = shfl_up(i1, d), y2 = shfl_up(i2, d);
+        if (lane >= d) { i1 += y1; i2 += y2; }
+    }
+    if (lane == 31) { tmp[warp] = i1; tmp[34 + warp] = i2; }
+    __syncthreads();
+    if (warp == 0) {
+        const uint64_t w1 = lane < nw ? tmp[lane] : 0ull, w2 = lane < nw ? tmp[34 + lane] : 0ull;
+        uint64_t a1 = w1, a2 = w2;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint64_t y1 = shfl_up(a1, d), y2 = shfl_up(a2, d);
+            if (lane >= d) { a1 += y1; a2 += y2; }
+        }
+        if (lane < nw) { tmp[lane] = a1 - w1; tmp[34 + lane] = a2 - w2; }
+        if (lane == nw - 1) { tmp[32] = a1; tmp[34 + 32] = a2; }
+    }
+    __syncthreads();
+    e1 = tmp[warp] + (i1 - x1);
+    e2 = tmp[34 + warp] + (i2 - x2);
+    t1 = tmp[32];
+    t2 = tmp[34 + 32];
+}
+
+// Slot counters are read in per-thread runs of consecutive slots: one padding word per 32 keeps those
+// reads free of bank conflicts.
+__device__ __forceinline__ int slot_pad(int s) { return s + (s >> 5); }
+
+struct SumShared {
+    unsigned int fill;        // nodes gathered so far
+    unsigned int nlong;       // long runs noted for the cooperative pass
+    unsigned int carryC;      // rows that have an element before the bucket
+    unsigned int pad;
+    unsigned long long carryS;   // sum of those elements
+};
+
+constexpr int SUM_SHORT = 4;          // runs of up to this many elements are gathered by the row's own thread
+
+// Dynamic shared memory: gathered nodes [scap] | nodes in time order [scap] (before the sort: the list of
+// long runs) | slot counters [scap + scap / 32 + 1] | rank of each gathered node inside its slot [scap].
+__global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, int R, int B, InstMeta *meta, FilterBufs F,
                                                      int nres, SegResult *seg) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
-    __shared__ uint64_t tmp[34];
+    __shared__ uint64_t tmpA[68], tmpB[68];
     __shared__ unsigned int sstatus;
     __shared__ InstMeta sM;
-    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
-    const int NG = nt / G, gi = tid / G, g = tid % G;
-    const int cap = F.scap;
-    Key<uint32_t> *keys = (Key<uint32_t> *)smem;
-    const BatchWS<uint32_t> ws{keys, keys + cap, (uint32_t *)(keys + 2 * (size_t)cap), cap};
+    __shared__ SumShared sh;
+    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+    const int cap = F.scap, nslots = max(32, cap / 2);
+    Key<uint32_t> *in = (Key<uint32_t> *)smem, *out = in + cap;
+    uint32_t *cnt = (uint32_t *)(out + cap);               // [slot_pad(nslots) + 1]: the last one closes the last slot
+    uint16_t *rk = (uint16_t *)(cnt + slot_pad(cap) + 2);
+    uint2 *longs = (uint2 *)out;                                  // (row | start << 16, end | position << 16)
+    const BatchWS<uint32_t> ws{in, out, cnt, cap};
     const bool single = F.scells == 0;
+    const int per = max(1, nslots / nt);
+    const int s0 = min(tid * per, nslots), s1 = min(s0 + per, nslots);
     for (int item = blockIdx.x; item < F.stiles * B; item += gridDim.x) {
         const int b = item / F.stiles, t = item - b * F.stiles;
         __syncthreads();                                          // shared state of the previous item is done with
@@ -1195,48 +1260,126 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
         const int64_t *inst = ts + (size_t)b * n * R;
         const uint32_t tminlo = (uint32_t)(uint64_t)M.tmin - 1u;
         const uint16_t *tab = single ? nullptr : F.itab + ((size_t)b * F.stiles + t) * n * 16;
+        const uint32_t *bnd = single ? nullptr : F.bnd + (size_t)b * ((size_t)F.stiles * TILE_BK + 1) + (size_t)t * TILE_BK;
         const int j1 = min(TILE_BK, (int)M.count - t * TILE_BK);  // buckets of this tile
         uint64_t bd = ~0ull, bt = ~0ull;
         bool over = false;
-        for (int j = 0; j < j1 && !over; ++j) {
-            // runs [s, e) of this group's rows: element count, and the carry-in from the runs' predecessors
-            uint32_t mycnt = 0, myC = 0;
+        for (int j = 0; j < j1; ++j) {
+            for (int s = tid; s <= slot_pad(nslots); s += nt) cnt[s] = 0;
+            if (tid == 0) { sh.fill = 0; sh.nlong = 0; sh.carryC = 0; sh.carryS = 0; }
+            // times of the bucket lie in [lo, hi): slot = ((T - lo) * scale) >> 32 < nslots, monotone in T
+            const uint32_t lo = single ? 1u : __ldg(bnd + j);
+            const uint64_t hi = single ? M.tend + 1 : min((uint64_t)__ldg(bnd + j + 1), M.tend + 1);
+            const uint32_t scale = (uint32_t)min((uint64_t)0xffffffffu, ((uint64_t)nslots << 32) / max((uint64_t)1, hi - (uint64_t)lo));
+            __syncthreads();
+            // K2 and the counting half of the sort.  A row's run [s, e) of the bucket: short runs are gathered
+            // by the row's thread (one round of independent loads), long ones are noted for whole warps.
             uint64_t myS = 0;
-            if (g == 0) {
-                for (int r = gi; r < n; r += NG) {
-                    const int s = single ? 0 : (int)__ldg(tab + (size_t)r * 16 + j);
-                    const int e = single ? R : (int)__ldg(tab + (size_t)r * 16 + j + 1);
-                    mycnt += (uint32_t)(e - s);
-                    if (s > 0) { myS += (uint32_t)(uint64_t)ldg64(inst + (size_t)r * R + s - 1) - tminlo; ++myC; }
-                }
-            }
-            uint64_t totcc, totS;
-            const uint64_t offcc = block_scan_excl<uint64_t>(((uint64_t)myC << 32) | mycnt, OpAdd(), 0ull, tmp, &totcc);
-            block_scan_excl<uint64_t>(myS, OpAdd(), 0ull, tmp, &totS);
-            const uint32_t m = (uint32_t)totcc;
-            if (m > (uint32_t)cap) { over = true; break; }
-            uint32_t o = (uint32_t)__shfl_sync(FULL, (uint32_t)offcc, lane - g);
-            for (int r = gi; r < n; r += NG) {
+            uint32_t myC = 0;
+            for (int r = tid; r < n; r += nt) {
                 const int s = single ? 0 : (int)__ldg(tab + (size_t)r * 16 + j);
                 const int e = single ? R : (int)__ldg(tab + (size_t)r * 16 + j + 1);
+                const int c = e - s;
                 const int64_t *rp = inst + (size_t)r * R;
-                for (int i = s + g; i < e; i += G) {
+                uint32_t v[SUM_SHORT + 1];
+                v[0] = s > 0 ? (uint32_t)(uint64_t)ldg64(rp + s - 1) - tminlo : 0u;
+#pragma unroll
+                for (int k = 0; k < SUM_SHORT; ++k) v[k + 1] = k < c && c <= SUM_SHORT ? (uint32_t)(uint64_t)ldg64(rp + s + k) - tminlo : 0u;
+                if (s > 0) { myS += v[0]; ++myC; }
+                if (c <= 0) continue;
+                const uint32_t o = atomicAdd(&sh.fill, (uint32_t)c);
+                if (o + (uint32_t)c > (uint32_t)cap) continue;    // the bucket does not fit: noticed below
+                if (c <= SUM_SHORT) {
+#pragma unroll
+                    for (int k = 0; k < SUM_SHORT; ++k) {
+                        if (k < c) {
+                            const uint32_t T = v[k + 1];
+                            in[o + k] = Key<uint32_t>::make(T, T - v[k]);
+                            rk[o + k] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
+                        }
+                    }
+                } else {
+                    longs[atomicAdd(&sh.nlong, 1u)] = make_uint2((uint32_t)r | ((uint32_t)s << 16), (uint32_t)e | (o << 16));
+                }
+            }
+            myS = warp_reduce(myS, OpAdd());
+            myC = warp_reduce(myC, OpAdd());
+            if (lane == 0 && myC) { atomicAdd(&sh.carryS, (unsigned long long)myS); atomicAdd(&sh.carryC, myC); }
+            __syncthreads();
+            const uint32_t m = sh.fill;
+            if (m > (uint32_t)cap) { over = true; break; }         // uniform over the block
+            const int nlong = (int)sh.nlong;
+            uint64_t cS = sh.carryS;
+            uint32_t cC = sh.carryC;
+            if (m == 0) continue;
+            for (int w = warp; w < nlong; w += nw) {
+                const uint2 d = longs[w];
+                const int r = (int)(d.x & 0xffffu), s = (int)(d.x >> 16), e = (int)(d.y & 0xffffu);
+                const uint32_t o = d.y >> 16;
+                const int64_t *rp = inst + (size_t)r * R;
+                for (int i = s + lane; i < e; i += 32) {
                     const uint32_t T = (uint32_t)(uint64_t)ldg64(rp + i) - tminlo;
                     const uint32_t pv = i > 0 ? (uint32_t)(uint64_t)ldg64(rp + i - 1) - tminlo : 0u;
-                    keys[o + (uint32_t)(i - s)] = Key<uint32_t>::make(T, T - pv);
+                    const uint32_t pos = o + (uint32_t)(i - s);
+                    in[pos] = Key<uint32_t>::make(T, T - pv);
+                    rk[pos] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
                 }
-                o += (uint32_t)(e - s);
             }
             __syncthreads();
-            uint64_t cS = totS;
-            uint32_t cC = (uint32_t)(totcc >> 32);
-            run_batch<uint32_t, ZL_OBJ_SUM>(ws, (int)m, (uint32_t)M.t0, n, tmp, (uint32_t)0, cS, cC, bd, bt);
+            // slot counts -> slot starts
+            uint32_t loc = 0, big = 0;
+            for (int s = s0; s < s1; ++s) { const uint32_t c = cnt[slot_pad(s)]; loc += c; big |= c > (uint32_t)SLOT_MAX; }
+            uint32_t tot;
+            uint32_t run = block_scan_excl<uint32_t>(loc, OpAdd(), 0u, (uint32_t *)tmpB, &tot);
+            if (__syncthreads_or((int)big)) {
+                // many equal or nearly equal times: the general batch routine (comparison network) takes the gathered nodes
+                run_batch<uint32_t, ZL_OBJ_SUM>(ws, (int)m, (uint32_t)M.t0, n, tmpA, (uint32_t)0, cS, cC, bd, bt);
+                continue;
+            }
+            for (int s = s0; s < s1; ++s) { const uint32_t c = cnt[slot_pad(s)]; cnt[slot_pad(s)] = run; run += c; }
+            if (tid == 0) cnt[slot_pad(nslots)] = m;
+            __syncthreads();
+            // nodes grouped by slot ...
+            for (uint32_t q = tid; q < m; q += nt) {
+                const Key<uint32_t> k = in[q];
+                out[cnt[slot_pad((int)min(__umulhi(k.t() - lo, scale), (uint32_t)nslots - 1u))] + rk[q]] = k;
+            }
+            __syncthreads();
+            // ... then every node to its rank among the few nodes of its slot: `in` becomes the bucket in time order (K1)
+            for (uint32_t q = tid; q < m; q += nt) {
+                const Key<uint32_t> k = out[q];
+                const int sl = (int)min(__umulhi(k.t() - lo, scale), (uint32_t)nslots - 1u);
+                const uint32_t sb = cnt[slot_pad(sl)], se = cnt[slot_pad(sl + 1)];
+                uint32_t rank = sb;
+                for (uint32_t i = sb; i < se; ++i) { const uint64_t w = out[i].w; rank += w < k.w || (w == k.w && i < q); }
+                in[rank] = k;
+            }
+            __syncthreads();
+            // K3 (sums of delta and of the first flags, carry-in from the runs' predecessors) and K4
+            const int ipt = (int)((m + nt - 1) / nt);
+            const int k0 = min((uint32_t)(tid * ipt), m), k1 = min((uint32_t)(k0 + ipt), m);
+            uint64_t ls = 0, lc = 0;
+            for (int k = k0; k < k1; ++k) { const Key<uint32_t> x = in[k]; ls += x.v(); lc += x.v() == x.t(); }
+            uint64_t sS, sC, tS, tC;
+            block_scan_add2(ls, lc, sS, sC, tS, tC, tmpA);
+            sS += cS;
+            uint32_t c = (uint32_t)sC + cC;
+            for (int k = k0; k < k1; ++k) {
+                const uint32_t T = in[k].t(), dl = in[k].v();
+                sS += dl;                                  // sum over started workers of their latest element
+                c += dl == T;                              // a first element carries delta == T (previous = 0)
+                if (c == (uint32_t)n) {
+                    const uint64_t w = (uint64_t)n * (uint64_t)T - sS;
+                    if (w < bd || (w == bd && (uint64_t)T < bt)) { bd = w; bt = T; }
+                }
+            }
         }
-        if (over) {                                               // uniform over the block
+        __syncthreads();
+        if (over) {
             if (tid == 0) { meta[b].overflow = 1; F.flags[1] = 1; }
             continue;
         }
-        block_best_to_result(bd, bt, ZL_OK, tmp, &sstatus, seg[(size_t)b * nres + t]);
+        block_best_to_result(bd, bt, ZL_OK, tmpA, &sstatus, seg[(size_t)b * nres + t]);
     }
 }
 
@@ -1704,22 +1847,24 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
                    (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg, q.B);
     } else if (sumfast) {
         const bool single = fb.scells == 0;
-        launch_dep(!((q.pdl_off >> 1) & 1), zl::k_sum_plan, dim3(q.B), dim3(single ? 32 : 1024), 0, st, q.ts, q.n, q.R, q.meta, fb);
+        const size_t nb1 = (size_t)fb.stiles * zl::TILE_BK + 1;
+        launch_dep(!((q.pdl_off >> 1) & 1), zl::k_sum_plan, dim3(q.B), dim3(single ? 32 : 1024), single ? 0 : ((size_t)fb.scells + 1) * 8 + nb1 * 4, st,
+                   q.ts, q.n, q.R, q.meta, fb);
         if (!single) {
             const int nw = 8;
             const int row_blocks = std::max(1, std::min((q.n + nw - 1) / nw, (32 * q.num_sms + q.B - 1) / q.B));
-            launch_dep(!((q.pdl_off >> 2) & 1), zl::k_sum_index, dim3(row_blocks, q.B), dim3(32 * nw), ((size_t)fb.stiles * zl::TILE_BK + 1) * 4, st, q.ts, q.n, q.R,
+            launch_dep(!((q.pdl_off >> 2) & 1), zl::k_sum_index, dim3(row_blocks, q.B), dim3(32 * nw), nb1 * 4, st, q.ts, q.n, q.R,
                        (const zl::InstMeta *)q.meta, fb);
         }
         if (ev) cudaEventRecord(ev[2], st);
         const long long N = (long long)q.n * q.R;
-        int bthreads = single ? (int)std::max<long long>(64, std::min<long long>(1024, pow2_ceil((int)((N + 3) / 4))))
+        int bthreads = single ? (int)std::max<long long>(64, std::min<long long>(1024, pow2_ceil((int)((N + 7) / 8))))
                               : (fb.scap > 4096 ? 1024 : 512);
         if (q.tail_threads) bthreads = q.tail_threads;
-        const int G = std::max(1, std::min(32, pow2_floor(std::max(1, bthreads / q.n))));
         const int items = fb.stiles * q.B;
-        launch_dep(!((q.pdl_off >> 3) & 1), zl::k_sum_buckets, dim3(std::min(items, 32 * q.num_sms)), dim3(bthreads), (size_t)fb.scap * 20, st,
-                   q.ts, q.n, q.R, q.B, G, q.meta, fb, q.nres, q.seg);
+        const size_t bsmem = (size_t)fb.scap * 18 + ((size_t)fb.scap + fb.scap / 32 + 2) * 4;
+        launch_dep(!((q.pdl_off >> 3) & 1), zl::k_sum_buckets, dim3(std::min(items, 32 * q.num_sms)), dim3(bthreads), bsmem, st,
+                   q.ts, q.n, q.R, q.B, q.meta, fb, q.nres, q.seg);
     } else if (ev) {
         cudaEventRecord(ev[2], st);
     }
@@ -1748,6 +1893,7 @@ cudaError_t raise_shared_memory_limits() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_tail, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_buckets, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_plan, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     return e;
 }
 
@@ -1862,13 +2008,12 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
             f.sM = f.scap / 16 * 11;
             const long long nbk = N / f.sM + 1;
             f.stiles = (int)((nbk + zl::TILE_BK - 1) / zl::TILE_BK);
-            f.scells = (int)std::max<long long>(1024, std::min<long long>(1 << 16, pow2_ceil((int)std::min<long long>(N / 64, 1 << 20))));
+            f.scells = (int)std::max<long long>(1024, std::min<long long>(1 << 14, pow2_ceil((int)std::min<long long>(N / 64, 1 << 20))));
             on = nbk <= 12000 && cfg->lookahead_R <= 65535;       // boundaries fit shared memory, row indices are 16-bit
         }
         if (on) {
             const size_t nb1 = (size_t)f.stiles * zl::TILE_BK + 1;
-            const size_t sizes[4] = {mb * nb1 * 4, mb * ((size_t)f.scells + 1 + nb1) * 8,
-                                     f.scells ? mb * f.stiles * cfg->n_workers * 32 : 64, 64};
+            const size_t sizes[4] = {mb * nb1 * 4, 64, f.scells ? mb * f.stiles * cfg->n_workers * 32 : 64, 64};
             void **ptrs[4] = {(void **)&f.bnd, (void **)&f.cellacc, (void **)&f.itab, (void **)&f.flags};
             for (int i = 0; i < 4; ++i) {
                 if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
