@@ -617,7 +617,17 @@ __device__ void run_batch(const BatchWS<K> &ws, int m, K t0, int n, uint64_t *tm
                           uint32_t &carryC, uint64_t &bd, uint64_t &bt) {
     if (m == 0) return;
     const Key<K> *keys;
-    if (m <= 256) {
+    if (m <= 128) {
+        // very small batches: every node counts the nodes that come before it (one barrier)
+        for (int q = threadIdx.x; q < m; q += blockDim.x) {
+            const Key<K> k = ws.in[q];
+            int rank = 0;
+            for (int i = 0; i < m; ++i) { const Key<K> o = ws.in[i]; rank += (k > o) || (!(o > k) && i < q); }
+            ws.out[rank] = k;
+        }
+        __syncthreads();
+        keys = ws.out;
+    } else if (m <= 256) {
         // small batches: the comparison network (mostly warp-local steps) beats the bookkeeping of the slot sort
         int P2 = 64;
         while (P2 < m) P2 <<= 1;
@@ -670,32 +680,32 @@ __device__ void run_batch(const BatchWS<K> &ws, int m, K t0, int n, uint64_t *tm
     __syncthreads();
 }
 
-// Block minimum of (objective, time) over the per-thread bests -> out.  red: 32 shared words.
+// Block minimum of (objective, time), compared as a pair, over the per-thread bests -> out.  red: 32 shared
+// 64-bit words that nobody reads any more; every thread calls; two barriers.
 __device__ void block_best_to_result(uint64_t bd, uint64_t bt, uint32_t status, uint64_t *red, unsigned int *sstatus,
                                      SegResult &out) {
-    const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = (blockDim.x + 31) >> 5;
+    __shared__ uint64_t red_t[32];
     for (int d = 16; d > 0; d >>= 1) {
         const uint64_t od = shfl_xor(bd, d), ot = shfl_xor(bt, d);
         if (od < bd || (od == bd && ot < bt)) { bd = od; bt = ot; }
     }
-    __syncthreads();
-    if (lane == 0) red[tid >> 5] = bd;
-    __syncthreads();
-    // two steps: the minimum objective, then the minimum time among its holders
-    uint64_t gd = ~0ull;
-    for (int w = 0; w < (nt >> 5); ++w) gd = min(gd, red[w]);
-    __syncthreads();
-    if (lane == 0) red[tid >> 5] = bd == gd ? bt : ~0ull;
-    __syncthreads();
-    uint64_t gt = ~0ull;
-    for (int w = 0; w < (nt >> 5); ++w) gt = min(gt, red[w]);
+    if (lane == 0) { red[warp] = bd; red_t[warp] = bt; }
     if (status != ZL_OK) atomicMax(sstatus, status);
     __syncthreads();
-    if (tid == 0) {
-        out.d = gd; out.t = gt;
-        out.valid = gd != ~0ull || gt != ~0ull;
-        out.status = (int32_t)*sstatus;
+    if (warp == 0) {
+        uint64_t gd = lane < nw ? red[lane] : ~0ull, gt = lane < nw ? red_t[lane] : ~0ull;
+        for (int d = 16; d > 0; d >>= 1) {
+            const uint64_t od = shfl_xor(gd, d), ot = shfl_xor(gt, d);
+            if (od < gd || (od == gd && ot < gt)) { gd = od; gt = ot; }
+        }
+        if (lane == 0) {
+            out.d = gd; out.t = gt;
+            out.valid = gd != ~0ull || gt != ~0ull;
+            out.status = (int32_t)*sstatus;
+        }
     }
+    __syncthreads();
 }
 
 // ------------------------------------------------------------------------------ sweep
@@ -1384,7 +1394,9 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
 }
 
 // Index of the last element of a sorted row that is <= bar (-1 if none).  Rows are close to arithmetic, so the
-// position is first guessed from the row's end points, bracketed by doubling steps around the guess, then bisected.
+// position is first guessed from the row's end points.  Eight probes around the guess, eight elements apart and
+// loaded together, then the seven elements between the two probes that bracket bar, loaded together: three
+// rounds of loads in the usual case.  A guess that is further off is bracketed by doubling steps and bisected.
 __device__ int last_index_not_after(const int64_t *row, int R, int64_t bar) {
     const int64_t e0 = ldg64(row), eR = ldg64(row + R - 1);
     if (bar < e0) return -1;
@@ -1393,15 +1405,37 @@ __device__ int last_index_not_after(const int64_t *row, int R, int64_t bar) {
     int lo, hi;
     int g = (int)((double)(bar - e0) * (double)(R - 1) / (double)(eR - e0));
     g = max(0, min(g, R - 2));
-    if (ldg64(row + g) <= bar) {
-        lo = g + 1; hi = R - 1;
-        for (int step = 1; lo < hi; step <<= 1) {
-            const int q = min(lo + step - 1, hi - 1);
+    {
+        constexpr int S = 8, P = 8;                       // probes at g + S * (k - P/2), clamped to the row
+        int64_t pv[P];
+        int pi[P];
+#pragma unroll
+        for (int k = 0; k < P; ++k) { pi[k] = max(0, min(R - 1, g + S * (k - P / 2))); pv[k] = ldg64(row + pi[k]); }
+        lo = 1; hi = R - 1;
+#pragma unroll
+        for (int k = 0; k < P; ++k) {
+            if (pv[k] <= bar) lo = max(lo, pi[k] + 1); else hi = min(hi, pi[k]);
+        }
+        if (hi - lo <= S - 1) {                            // bracketed between two neighbouring probes
+            int64_t wv[S - 1];
+#pragma unroll
+            for (int k = 0; k < S - 1; ++k) wv[k] = ldg64(row + min(lo + k, R - 1));
+            int c = 0;
+#pragma unroll
+            for (int k = 0; k < S - 1; ++k) c += (lo + k < hi && wv[k] <= bar) ? 1 : 0;   // sorted: a prefix of the window
+            return lo + c - 1;
+        }
+    }
+    // the probes did not enclose bar closely: doubling steps from the nearer end of the bracket, then bisection
+    if (lo > 1) {                                          // everything probed was <= bar: search upwards from lo
+        const int top = hi;
+        for (int step = 16; lo < hi; step <<= 1) {
+            const int q = min(lo + step - 1, top - 1);
+            if (q < lo) break;
             if (ldg64(row + q) <= bar) lo = q + 1; else { hi = q; break; }
         }
-    } else {
-        hi = g; lo = 1;
-        for (int step = 1; lo < hi; step <<= 1) {
+    } else {                                               // everything probed was > bar: search downwards from hi
+        for (int step = 16; lo < hi; step <<= 1) {
             const int q = max(hi - step, lo);
             if (ldg64(row + q) > bar) hi = q; else { lo = q + 1; break; }
         }
