@@ -1242,6 +1242,7 @@ constexpr int SUM_SHORT = 4;          // runs of up to this many elements are ga
 
 // Dynamic shared memory: gathered nodes [scap] | nodes in time order [scap] (before the sort: the list of
 // long runs) | slot counters [scap + scap / 32 + 1] | rank of each gathered node inside its slot [scap].
+template <int OBJ>
 __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, int R, int B, InstMeta *meta, FilterBufs F,
                                                      int nres, SegResult *seg) {
     grid_dep_wait();
@@ -1291,10 +1292,12 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
                 const int e = single ? R : (int)__ldg(tab + (size_t)r * 16 + j + 1);
                 const int c = e - s;
                 const int64_t *rp = inst + (size_t)r * R;
-                uint32_t v[SUM_SHORT + 1];
+                uint32_t v[SUM_SHORT + 2];                        // predecessor, the run, and (RANGE) the element after it
                 v[0] = s > 0 ? (uint32_t)(uint64_t)ldg64(rp + s - 1) - tminlo : 0u;
 #pragma unroll
                 for (int k = 0; k < SUM_SHORT; ++k) v[k + 1] = k < c && c <= SUM_SHORT ? (uint32_t)(uint64_t)ldg64(rp + s + k) - tminlo : 0u;
+                v[SUM_SHORT + 1] = 0xffffffffu;
+                if (OBJ == ZL_OBJ_RANGE && c > 0 && c <= SUM_SHORT && e < R) v[SUM_SHORT + 1] = (uint32_t)(uint64_t)ldg64(rp + e) - tminlo;
                 if (s > 0) { myS += v[0]; ++myC; }
                 if (c <= 0) continue;
                 const uint32_t o = atomicAdd(&sh.fill, (uint32_t)c);
@@ -1304,7 +1307,8 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
                     for (int k = 0; k < SUM_SHORT; ++k) {
                         if (k < c) {
                             const uint32_t T = v[k + 1];
-                            in[o + k] = Key<uint32_t>::make(T, T - v[k]);
+                            // payload: SUM T minus the row's previous element, RANGE the row's next element
+                            in[o + k] = Key<uint32_t>::make(T, OBJ == ZL_OBJ_SUM ? T - v[k] : k + 1 < c ? v[k + 2] : v[SUM_SHORT + 1]);
                             rk[o + k] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
                         }
                     }
@@ -1329,9 +1333,11 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
                 const int64_t *rp = inst + (size_t)r * R;
                 for (int i = s + lane; i < e; i += 32) {
                     const uint32_t T = (uint32_t)(uint64_t)ldg64(rp + i) - tminlo;
-                    const uint32_t pv = i > 0 ? (uint32_t)(uint64_t)ldg64(rp + i - 1) - tminlo : 0u;
+                    uint32_t pay;
+                    if (OBJ == ZL_OBJ_SUM) pay = T - (i > 0 ? (uint32_t)(uint64_t)ldg64(rp + i - 1) - tminlo : 0u);
+                    else pay = i + 1 < R ? (uint32_t)(uint64_t)ldg64(rp + i + 1) - tminlo : 0xffffffffu;
                     const uint32_t pos = o + (uint32_t)(i - s);
-                    in[pos] = Key<uint32_t>::make(T, T - pv);
+                    in[pos] = Key<uint32_t>::make(T, pay);
                     rk[pos] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
                 }
             }
@@ -1343,7 +1349,7 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
             uint32_t run = block_scan_excl<uint32_t>(loc, OpAdd(), 0u, (uint32_t *)tmpB, &tot);
             if (__syncthreads_or((int)big)) {
                 // many equal or nearly equal times: the general batch routine (comparison network) takes the gathered nodes
-                run_batch<uint32_t, ZL_OBJ_SUM>(ws, (int)m, (uint32_t)M.t0, n, tmpA, (uint32_t)0, cS, cC, bd, bt);
+                run_batch<uint32_t, OBJ>(ws, (int)m, (uint32_t)M.t0, n, tmpA, (uint32_t)0, cS, cC, bd, bt);
                 continue;
             }
             for (int s = s0; s < s1; ++s) { const uint32_t c = cnt[slot_pad(s)]; cnt[slot_pad(s)] = run; run += c; }
@@ -1368,19 +1374,37 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
             // K3 (sums of delta and of the first flags, carry-in from the runs' predecessors) and K4
             const int ipt = (int)((m + nt - 1) / nt);
             const int k0 = min((uint32_t)(tid * ipt), m), k1 = min((uint32_t)(k0 + ipt), m);
-            uint64_t ls = 0, lc = 0;
-            for (int k = k0; k < k1; ++k) { const Key<uint32_t> x = in[k]; ls += x.v(); lc += x.v() == x.t(); }
-            uint64_t sS, sC, tS, tC;
-            block_scan_add2(ls, lc, sS, sC, tS, tC, tmpA);
-            sS += cS;
-            uint32_t c = (uint32_t)sC + cC;
-            for (int k = k0; k < k1; ++k) {
-                const uint32_t T = in[k].t(), dl = in[k].v();
-                sS += dl;                                  // sum over started workers of their latest element
-                c += dl == T;                              // a first element carries delta == T (previous = 0)
-                if (c == (uint32_t)n) {
-                    const uint64_t w = (uint64_t)n * (uint64_t)T - sS;
-                    if (w < bd || (w == bd && (uint64_t)T < bt)) { bd = w; bt = T; }
+            if (OBJ == ZL_OBJ_SUM) {
+                uint64_t ls = 0, lc = 0;
+                for (int k = k0; k < k1; ++k) { const Key<uint32_t> x = in[k]; ls += x.v(); lc += x.v() == x.t(); }
+                uint64_t sS, sC, tS, tC;
+                block_scan_add2(ls, lc, sS, sC, tS, tC, tmpA);
+                sS += cS;
+                uint32_t c = (uint32_t)sC + cC;
+                for (int k = k0; k < k1; ++k) {
+                    const uint32_t T = in[k].t(), dl = in[k].v();
+                    sS += dl;                              // sum over started workers of their latest element
+                    c += dl == T;                          // a first element carries delta == T (previous = 0)
+                    if (c == (uint32_t)n) {
+                        const uint64_t w = (uint64_t)n * (uint64_t)T - sS;
+                        if (w < bd || (w == bd && (uint64_t)T < bt)) { bd = w; bt = T; }
+                    }
+                }
+            } else {
+                // RANGE (single-bucket instances only: nothing is carried in): prefix max of next, d = max(T, t0, PM) - T
+                uint32_t lmax = 0;
+                for (int k = k0; k < k1; ++k) lmax = max(lmax, in[k].v());
+                uint32_t totm;
+                uint32_t pm = block_scan_excl<uint32_t>(lmax, OpMax(), 0u, (uint32_t *)tmpA, &totm);
+                const uint32_t t0 = (uint32_t)M.t0;
+                for (int k = k0; k < k1; ++k) {
+                    const uint32_t T = in[k].t();
+                    const uint32_t g = max(max(T, t0), pm);   // max(Z) of the best Z whose minimum is this element
+                    if (g != 0xffffffffu) {
+                        const uint64_t d = (uint64_t)(g - T);
+                        if (d < bd || (d == bd && (uint64_t)T < bt)) { bd = d; bt = T; }
+                    }
+                    pm = max(pm, in[k].v());
                 }
             }
         }
@@ -1538,9 +1562,10 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
                                                   int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
     grid_dep_wait();
     const int b = blockIdx.y, tid = threadIdx.x;
+    // filter: 0 only the segment sweep ran, 1 the RANGE filter route, 2 the bucket route
     if (filter && F.flags[2] == 0) return;                        // k_tail finished every instance of this call
     const InstMeta M = meta[b];
-    if (objective == ZL_OBJ_RANGE && M.status == ZL_OK && handled_by_filter(M, filter) && tail_instance(M)) return;   // finished by k_tail
+    if (filter == 1 && M.status == ZL_OK && handled_by_filter(M, filter) && tail_instance(M)) return;   // finished by k_tail
     __shared__ uint64_t red[34];
     __shared__ unsigned int sstatus;
     __shared__ SegResult best;
@@ -1550,7 +1575,7 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
     uint32_t st = M.status;
     if (st == ZL_OK) {
         const int used = !handled_by_filter(M, filter) ? nseg
-                         : objective == ZL_OBJ_SUM ? (int)M.count2                      // bucket route: one result per tile
+                         : filter == 2 ? (int)M.count2                                  // bucket route: one result per tile
                          : tail_instance(M) ? 1 : (F.nbk + bucket_group(F, M.count2) - 1) / bucket_group(F, M.count2);
         for (int s = tid; s < used; s += blockDim.x) {
             const SegResult r = seg[(size_t)b * nres + s];
@@ -1839,7 +1864,8 @@ void launch_dep(bool early, void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
 
 void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_t *ev) {
     const bool filter = q.fb.table != nullptr && q.objective == ZL_OBJ_RANGE;
-    const bool sumfast = q.fb.flags != nullptr && q.fb.scap != 0 && q.objective == ZL_OBJ_SUM;
+    // the bucket route: every SUM shape it supports, and RANGE instances small enough to be a single bucket
+    const bool sumfast = q.fb.flags != nullptr && q.fb.scap != 0 && (q.objective == ZL_OBJ_SUM || q.fb.table == nullptr);
     zl::FilterBufs fb = q.fb;
     if (!filter && !sumfast) memset(&fb, 0, sizeof(fb));
     if (ev) cudaEventRecord(ev[0], st);
@@ -1897,8 +1923,12 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         if (q.tail_threads) bthreads = q.tail_threads;
         const int items = fb.stiles * q.B;
         const size_t bsmem = (size_t)fb.scap * 18 + ((size_t)fb.scap + fb.scap / 32 + 2) * 4;
-        launch_dep(!((q.pdl_off >> 3) & 1), zl::k_sum_buckets, dim3(std::min(items, 32 * q.num_sms)), dim3(bthreads), bsmem, st,
-                   q.ts, q.n, q.R, q.B, q.meta, fb, q.nres, q.seg);
+        if (q.objective == ZL_OBJ_SUM)
+            launch_dep(!((q.pdl_off >> 3) & 1), zl::k_sum_buckets<ZL_OBJ_SUM>, dim3(std::min(items, 32 * q.num_sms)), dim3(bthreads), bsmem, st,
+                       q.ts, q.n, q.R, q.B, q.meta, fb, q.nres, q.seg);
+        else
+            launch_dep(!((q.pdl_off >> 3) & 1), zl::k_sum_buckets<ZL_OBJ_RANGE>, dim3(std::min(items, 32 * q.num_sms)), dim3(bthreads), bsmem, st,
+                       q.ts, q.n, q.R, q.B, q.meta, fb, q.nres, q.seg);
     } else if (ev) {
         cudaEventRecord(ev[2], st);
     }
@@ -1916,7 +1946,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     if (ev) cudaEventRecord(ev[3], st);
     const int fthreads = std::max(32, std::min(256, pow2_ceil(q.n)));
     launch_dep(!((q.pdl_off >> 8) & 1), zl::k_finalize, dim3((q.n + fthreads - 1) / fthreads, q.B), dim3(fthreads), 0, st, q.ts, q.n, q.R, p.nseg, fb, q.nres, q.objective,
-                                                                  fast ? 1 : 0, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
+                                                                  filter ? 1 : sumfast ? 2 : 0, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
     if (ev) cudaEventRecord(ev[4], st);
 }
 
@@ -1926,7 +1956,8 @@ cudaError_t raise_shared_memory_limits() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_buckets, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_tail, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_buckets, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_buckets<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_buckets<ZL_OBJ_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_plan, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     return e;
 }
@@ -2009,7 +2040,9 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     const size_t meta_b = (size_t)cfg->max_batch * sizeof(zl::InstMeta);
     size_t filter_b = 0;
     h->nres = zl::MAX_SEGMENTS;
-    if (cfg->objective == ZL_OBJ_RANGE) {
+    // RANGE instances that fit one shared-memory batch are sorted whole by the bucket route; larger ones take the filter route
+    const bool range_small = cfg->objective == ZL_OBJ_RANGE && (long long)cfg->n_workers * cfg->lookahead_R <= 4096;
+    if (cfg->objective == ZL_OBJ_RANGE && !range_small) {
         const long long N = (long long)cfg->n_workers * cfg->lookahead_R;
         const size_t mb = (size_t)cfg->max_batch;
         zl::FilterBufs &f = h->fb;
@@ -2030,7 +2063,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
             filter_b += sizes[i];
         }
     }
-    if (cfg->objective == ZL_OBJ_SUM) {
+    if (cfg->objective == ZL_OBJ_SUM || range_small) {
         // bucket route: shared-memory batches of scap elements, buckets of about 11/16 of that
         const long long N = (long long)cfg->n_workers * cfg->lookahead_R;
         const size_t mb = (size_t)cfg->max_batch;
@@ -2177,8 +2210,8 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
 size_t zl_workspace_bytes(const zl_handle *h) { return h ? h->ws_bytes + h->staging_bytes : 0; }
 int32_t zl_launches_per_call(const zl_handle *h) {
     if (!h) return 0;
-    const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter;
-    const bool sumfast = h->cfg.objective == ZL_OBJ_SUM && !h->opt_no_filter && h->fb.scap != 0;
+    const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter && h->fb.table != nullptr;
+    const bool sumfast = !filter && !h->opt_no_filter && h->fb.scap != 0;
     return 3 + (filter ? 6 : 0) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
 }
 int32_t zl_segments_per_instance(const zl_handle *h, int32_t B) { return h && B >= 1 ? make_plan(h, B).nseg : 0; }

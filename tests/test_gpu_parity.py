@@ -196,7 +196,10 @@ def test_host_detected_errors():
         h.select_batched(ts)             # B > max_batch
     with pytest.raises(zl.ZipLineError):
         h.set_option("no_such_option", 1)
-    assert h.launches_per_call == 9 and h.workspace_bytes > 0
+    assert h.launches_per_call == 5 and h.workspace_bytes > 0      # tiny shape: prologue, plan, buckets, sweep, finalize
+    h2 = zl.ZipLine(64, 128, 2)
+    assert h2.launches_per_call == 9                                 # the filter route
+    h2.destroy()
     h.destroy()
 
 
