@@ -272,6 +272,7 @@ def main():
     e2e_steps = max(3, min(args.steps, 10))
     ms_e, _, _ = timed(h, e2e_steps, 3, host=True)
     e2e_value = world * nts / (ms_e / e2e_steps * 1e-3)
+    h_route = h.route
     h.destroy()
 
     if rank != 0:
@@ -282,10 +283,16 @@ def main():
     # ---- roofline of the dominant kernel (the sweep), algorithmic bytes = 8 per timestamp it must examine
     peak, peak_kind = measured_peak_gbs()
     lmin = ts_np[:, :, -1].min(axis=1)
-    examined = int((ts_np <= lmin[:, None, None]).sum()) if objective == 0 else nts
+    route = h_route                                  # 0 segment sweep only, 1 RANGE filter route, 2 bucket route
+    examined = int((ts_np <= lmin[:, None, None]).sum()) if route == 1 else nts
     def dominant(pr):
-        stages = {"k_prologue": pr["ms_prologue"], "k_filter": pr["ms_filter"],
-                  "k_tail+k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep": pr["ms_sweep"], "k_finalize": pr["ms_finalize"]}
+        if route == 1:
+            names = ("k_prologue", "k_filter", "k_tail+k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep", "k_finalize")
+        elif route == 2:
+            names = ("k_prologue", "k_sum_plan+k_sum_index", "k_sum_buckets+k_sweep", "k_finalize")
+        else:
+            names = ("k_prologue", "-", "k_sweep", "k_finalize")
+        stages = dict(zip(names, (pr["ms_prologue"], pr["ms_filter"], pr["ms_sweep"], pr["ms_finalize"])))
         name = max(stages, key=stages.get)
         return name, stages[name] / pr["calls"]
 
@@ -298,7 +305,7 @@ def main():
                 "traffic": recorded_traffic(f"{w.name}_{args.objective}_default_{dom}"),
                 "bytes_per_launch": examined * 8, "ms_per_launch": sweep_ms,
                 "bytes_model": "8 B per timestamp not after the first exhausted row (the search stops there)"
-                if objective == 0 else "8 B per timestamp"}
+                if route == 1 else "8 B per timestamp"}
     full = {"value": nts / (ms_f / steps_f * 1e-3), "unit": "timestamps/s", "ms_per_step": ms_f / steps_f,
             "roofline": {"bound": "hbm", "kernel": dom_f, "achieved": ach_f, "peak": peak, "unit": "GB/s",
                          "frac": ach_f / peak, "bytes_per_launch": nts * 8, "ms_per_launch": sweep_ms_f,
@@ -311,7 +318,8 @@ def main():
                "sample": f"{Bs} of {w.B} instances of {w.name}, sweep_window (sort + one pass), {dt:.1f} s wall"}
 
     cfg = workload_config(w, objective, world)
-    cfg.update({"selections_per_s": world * w.B / (ms_step * 1e-3), "early_stop": objective == 0,
+    cfg.update({"selections_per_s": world * w.B / (ms_step * 1e-3), "early_stop": route == 1,
+                "route": {0: "segment sweep", 1: "filter", 2: "buckets"}[route],
                 "examined_fraction": examined / nts, "segments_per_instance": None,
                 "kernel_ms": {k[3:]: prof[k] / prof["calls"] for k in ("ms_prologue", "ms_filter", "ms_sweep", "ms_finalize")},
                 "kernel_ms_full_sweep": {k[3:]: prof_f[k] / prof_f["calls"]

@@ -232,16 +232,18 @@ zl_status zl_destroy(zl_handle *h);
  * Diagnostic (no counterpart in the paper): for the last zl_select_batched on h and each of
  * its first B instances, how many elements passed the RANGE filter pass (h_filtered), how many of
  * those passed the refinement (h_refined), and whether a survivor list overflowed, in which case
- * the segment sweep handled the instance instead (h_overflow).  Host arrays of B uint32, any of
- * which may be NULL.  Synchronises the device.
+ * the segment sweep handled the instance instead (h_overflow).  On the bucket route (zl_route() == 2)
+ * the three arrays hold the instance's time buckets, its tiles of buckets, and whether a bucket
+ * outgrew its shared-memory batch (the segment sweep then handled the instance).  Host arrays of B
+ * uint32, any of which may be NULL.  Synchronises the device.
  */
 zl_status zl_filter_counts(zl_handle *h, int32_t B, uint32_t *h_filtered, uint32_t *h_refined, uint32_t *h_overflow);
 
 /* Tuning knobs of a handle (host side; take effect at the next call).
  * key: "threads" (128..1024, power of two), "lanes_per_row" (1..32, power of two),
  * "segments" (time segments per instance, >= 1), "round_factor" (percent of the
- * nominal elements per round), "no_filter" (1: RANGE skips the filter pass and sweeps
- * every instance by time segments), "filter_threads" / "filter_rows" (CTA size and rows per CTA of the
+ * nominal elements per round), "no_filter" (1: neither the RANGE filter route nor the bucket
+ * route is used; every instance is swept by time segments), "filter_threads" / "filter_rows" (CTA size and rows per CTA of the
  * filter pass), "prologue_threads" / "tail_threads" (CTA sizes of those kernels), "pdl_off" (bit k: launch the k-th kernel of the chain only after its predecessor has
  * finished instead of scheduling it early).  0 restores the built-in choice. */
 zl_status zl_set_option(zl_handle *h, const char *key, int32_t value);
@@ -251,6 +253,7 @@ const char *zl_status_string(zl_status s);
 size_t   zl_workspace_bytes(const zl_handle *h);      /* device scratch held by the handle      */
 int32_t  zl_launches_per_call(const zl_handle *h);    /* kernels one zl_select_batched enqueues  */
 int32_t  zl_segments_per_instance(const zl_handle *h, int32_t B);
+int32_t  zl_route(const zl_handle *h);                /* route of the handle's calls: 0 segment sweep only, 1 RANGE filter route, 2 bucket route */
 int32_t  zl_max_workers(void);                        /* largest supported n                     */
 int32_t  zl_trace_max_elements(void);                 /* largest n*R for zl_trace_batched        */
 int32_t  zl_last_cuda_error(const zl_handle *h);      /* cudaError_t of the last failed call     */

@@ -23,7 +23,7 @@ EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace
            "zl_segments_per_instance", "zl_max_workers", "zl_trace_max_elements", "zl_last_cuda_error",
            "zl_profile_begin", "zl_profile_read", "zl_profile_end",
            "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes", "zl_filter_counts",
-           "zl_predict_batched", "zl_predict_select_batched", "zl_gridscan_batched")
+           "zl_predict_batched", "zl_predict_select_batched", "zl_gridscan_batched", "zl_route")
 
 
 class zl_config(ctypes.Structure):
@@ -46,6 +46,8 @@ def _load() -> ctypes.CDLL:
     lib.zl_workspace_bytes.restype = ctypes.c_size_t
     lib.zl_launches_per_call.argtypes = [vp]
     lib.zl_segments_per_instance.argtypes = [vp, i32]
+    lib.zl_route.argtypes = [vp]
+    lib.zl_route.restype = ctypes.c_int
     lib.zl_last_cuda_error.argtypes = [vp]
     lib.zl_profile_begin.argtypes = [vp, i32]
     lib.zl_profile_read.argtypes = [vp, vp, vp]
@@ -211,6 +213,11 @@ class ZipLine:
     @property
     def launches_per_call(self) -> int:
         return lib.zl_launches_per_call(self._h)
+
+    @property
+    def route(self) -> int:
+        """0: segment sweep only, 1: RANGE filter route, 2: bucket route."""
+        return lib.zl_route(self._h)
 
     def segments_per_instance(self, B: int) -> int:
         return lib.zl_segments_per_instance(self._h, B)

@@ -16,7 +16,15 @@
 //               instances with many survivors: G at every fine time cell, drop what cannot matter,
 //               bucket by time, sort + scan + evaluate per group of buckets.
 //
-// SUM (sum_p (max(Z) - z_p)), and RANGE instances the filter route cannot take: the segment sweep.
+// SUM (sum_p (max(Z) - z_p)): every element matters, so the whole instance is put into time order, bucket by
+// bucket (the bucket route; also taken by RANGE instances small enough to be one shared-memory batch).
+//   k_sum_plan     bucket start times from the expected element density over the timeline.
+//   k_sum_index    one streaming pass: per row and bucket, the index of the row's first element in the bucket.
+//   k_sum_buckets  per bucket: gather the rows' runs (delta + first flag, or next), sort in shared memory,
+//                  scan with the carry-in the runs' predecessors give, evaluate, keep the first minimum.
+//
+// Instances neither fast route can take (time span of 2^32 us or more, an overflowing list or bucket): the
+// segment sweep.
 //   k_sweep     the timeline is cut into time segments.  A CTA walks its segment in rounds: every row
 //               advances a cursor over the elements inside the round's time window (the rows are
 //               sorted, so the n-way merge is a set of cursors), attaches the payload the scan needs
@@ -1031,7 +1039,9 @@ __global__ void __launch_bounds__(256) k_buckets(const InstMeta *meta, FilterBuf
 //                  (S = sum over rows of the last element before the bucket, cnt = rows that have one),
 //                  evaluates n*T - S where cnt == n (K4) and keeps the first minimum (K5, per tile).
 // A bucket that holds more than scap elements (rows far from arithmetic) sends its instance to the
-// segment sweep instead.
+// segment sweep instead.  An instance with n * R <= scap is a single bucket (no plan, no index table);
+// RANGE instances of that size take this route too: the payload of a node is then the same row's next
+// element and the scan is the exclusive prefix maximum, d = max(T, t0, PM) - T.
 constexpr int TILE_BK = 15;           // buckets per tile: 16 boundaries = 32 bytes per row and tile
 constexpr int SUM_FP = 12;            // fixed-point bits of the expected counts
 
@@ -1107,14 +1117,17 @@ __global__ void __launch_bounds__(1024) k_sum_plan(const int64_t *ts, int n, int
     const unsigned long long per_bucket = (unsigned long long)F.sM << SUM_FP;
     const uint32_t nbmax = (uint32_t)(F.stiles * TILE_BK);
     const uint32_t nbk = (uint32_t)max(1ull, min((unsigned long long)nbmax, (acc[cells] + per_bucket - 1) / per_bucket));
-    for (uint32_t c = tid; c < cells; c += nt) {
-        const unsigned long long lo = acc[c], hi = acc[c + 1];
-        if (hi == lo) continue;
-        unsigned long long k = max(1ull, (lo + per_bucket - 1) / per_bucket);
-        if (k >= nbk || k * per_bucket >= hi) continue;
-        const unsigned long long start = ((unsigned long long)c << 32) / cscale + 1, next = ((unsigned long long)(c + 1) << 32) / cscale + 1;
-        for (; k < nbk && k * per_bucket < hi; ++k)
-            bsm[k] = (uint32_t)min(0xfffffffeull, start + (k * per_bucket - lo) * (next - start) / (hi - lo));
+    // one thread per boundary (few): the cell in which the cumulated expectation passes k * sM, by bisection
+    for (uint32_t k = 1 + tid; k < nbk; k += nt) {
+        const unsigned long long target = (unsigned long long)k * per_bucket;      // < acc[cells]
+        uint32_t c0 = 0, c1 = cells - 1;                          // last cell with acc[c] <= target
+        while (c0 < c1) {
+            const uint32_t mid = (c0 + c1 + 1) >> 1;
+            if (acc[mid] <= target) c0 = mid; else c1 = mid - 1;
+        }
+        const unsigned long long lo = acc[c0], hi = acc[c0 + 1];  // lo <= target < hi
+        const unsigned long long start = ((unsigned long long)c0 << 32) / cscale + 1, next = ((unsigned long long)(c0 + 1) << 32) / cscale + 1;
+        bsm[k] = (uint32_t)min(0xfffffffeull, start + (target - lo) * (next - start) / max(1ull, hi - lo));
     }
     if (tid == 0) { bsm[0] = 0; bsm[nbk] = 0xffffffffu; }
     __syncthreads();
@@ -2213,6 +2226,11 @@ int32_t zl_launches_per_call(const zl_handle *h) {
     const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter && h->fb.table != nullptr;
     const bool sumfast = !filter && !h->opt_no_filter && h->fb.scap != 0;
     return 3 + (filter ? 6 : 0) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
+}
+int32_t zl_route(const zl_handle *h) {
+    if (!h || h->opt_no_filter) return 0;
+    if (h->cfg.objective == ZL_OBJ_RANGE && h->fb.table != nullptr) return 1;
+    return h->fb.scap != 0 ? 2 : 0;
 }
 int32_t zl_segments_per_instance(const zl_handle *h, int32_t B) { return h && B >= 1 ? make_plan(h, B).nseg : 0; }
 int32_t zl_last_cuda_error(const zl_handle *h) { return h ? h->last_cuda_error : 0; }
