@@ -315,6 +315,46 @@ def test_sum_routes_are_all_exercised_and_exact():
     assert_same(ts, 1, got)
 
 
+def test_sum_bucket_counts_around_tile_boundaries():
+    # instance sizes chosen so that the number of buckets walks across multiples of the tile size (15 buckets):
+    # the index table stores such a boundary twice, and the last tile may hold one bucket or fifteen
+    seen = set()
+    for k, R in enumerate((330, 352, 374, 396, 680, 704, 726, 1050)):
+        n = 120
+        ts = zi.generate(zi.CONFIGS["c3"].with_(B=2, n=n, R=R), first_instance=10 * k)
+        got, buckets, tiles, overflow = _sum_routes(ts)
+        assert (overflow == 0).all()
+        seen.update(int(b) % 15 for b in buckets)
+        assert_same(ts, 1, got)
+    assert len(seen) >= 4                      # several different fillings of the last tile were exercised
+
+
+def test_sum_buckets_with_heavy_ties_and_odd_shapes():
+    rng = np.random.default_rng(4242)
+    # many equal timestamps inside a bucket (slots fuller than the rank step allows: the comparison network takes over),
+    # rows of odd length, a row count that is not a multiple of the CTA's threads
+    for n, R, B, hi in ((77, 333, 3, 3), (130, 257, 2, 40), (513, 45, 2, 2000), (45, 1001, 2, 10 ** 6)):
+        inc = rng.integers(0, hi, size=(B, n, R))
+        ts = (rng.integers(0, 3 * hi, size=(B, n, 1)) + np.cumsum(inc, axis=2)).astype(np.int64)
+        got, buckets, tiles, overflow = _sum_routes(ts)
+        assert_same(ts, 1, got)
+
+
+def test_range_single_bucket_route_shapes():
+    # RANGE instances of at most 4096 timestamps are sorted whole by one CTA
+    rng = np.random.default_rng(99)
+    for n, R, B, hi in ((16, 64, 300, 10 ** 5), (4096, 1, 2, 1000), (1, 4096, 2, 50), (63, 65, 5, 7), (2, 2048, 3, 10 ** 9)):
+        inc = rng.integers(0, hi, size=(B, n, R))
+        ts = (rng.integers(0, 3 * hi, size=(B, n, 1)) + np.cumsum(inc, axis=2)).astype(np.int64)
+        h = zl.ZipLine(n, R, B, 0)
+        assert h.route == 2
+        h.destroy()
+        assert_same(ts, 0, gpu_select(ts, 0))
+    h = zl.ZipLine(64, 65, 1, 0)
+    assert h.route == 1                        # 4160 timestamps: the filter route
+    h.destroy()
+
+
 def test_sum_mixed_batch_of_routes():
     # a regular, an overflowing and a wide-span instance in one batch
     n, R = 128, 512
