@@ -1256,7 +1256,7 @@ constexpr int SUM_SHORT = 4;          // runs of up to this many elements are ga
 // Dynamic shared memory: gathered nodes [scap] | nodes in time order [scap] (before the sort: the list of
 // long runs) | slot counters [scap + scap / 32 + 1] | rank of each gathered node inside its slot [scap].
 template <int OBJ>
-__global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, int R, int B, InstMeta *meta, FilterBufs F,
+__global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, int R, int B, int early_stop, InstMeta *meta, FilterBufs F,
                                                      int nres, SegResult *seg) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
@@ -1292,8 +1292,10 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
             for (int s = tid; s <= slot_pad(nslots); s += nt) cnt[s] = 0;
             if (tid == 0) { sh.fill = 0; sh.nlong = 0; sh.carryC = 0; sh.carryS = 0; }
             // times of the bucket lie in [lo, hi): slot = ((T - lo) * scale) >> 32 < nslots, monotone in T
+            // RANGE: once some row's last element has passed no later Z is complete, so nodes after lmin are left out
+            const uint32_t tcut = OBJ == ZL_OBJ_RANGE && early_stop ? (uint32_t)M.lmin : 0xffffffffu;
             const uint32_t lo = single ? 1u : __ldg(bnd + j);
-            const uint64_t hi = single ? M.tend + 1 : min((uint64_t)__ldg(bnd + j + 1), M.tend + 1);
+            const uint64_t hi = single ? min(M.tend, (uint64_t)tcut) + 1 : min((uint64_t)__ldg(bnd + j + 1), M.tend + 1);
             const uint32_t scale = (uint32_t)min((uint64_t)0xffffffffu, ((uint64_t)nslots << 32) / max((uint64_t)1, hi - (uint64_t)lo));
             __syncthreads();
             // K2 and the counting half of the sort.  A row's run [s, e) of the bucket: short runs are gathered
@@ -1313,48 +1315,65 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
                 if (OBJ == ZL_OBJ_RANGE && c > 0 && c <= SUM_SHORT && e < R) v[SUM_SHORT + 1] = (uint32_t)(uint64_t)ldg64(rp + e) - tminlo;
                 if (s > 0) { myS += v[0]; ++myC; }
                 if (c <= 0) continue;
-                const uint32_t o = atomicAdd(&sh.fill, (uint32_t)c);
-                if (o + (uint32_t)c > (uint32_t)cap) continue;    // the bucket does not fit: noticed below
+                // SUM reserves the run's places in one step; RANGE appends node by node (it leaves nodes out)
+                const uint32_t o_run = OBJ == ZL_OBJ_SUM ? atomicAdd(&sh.fill, (uint32_t)c) : 0u;
+                if (o_run + (uint32_t)c > (uint32_t)cap) continue;   // the bucket does not fit: noticed below
                 if (c <= SUM_SHORT) {
 #pragma unroll
                     for (int k = 0; k < SUM_SHORT; ++k) {
-                        if (k < c) {
+                        if (k < c && v[k + 1] <= tcut) {
                             const uint32_t T = v[k + 1];
+                            const uint32_t o = OBJ == ZL_OBJ_SUM ? o_run + (uint32_t)k : atomicAdd(&sh.fill, 1u);
                             // payload: SUM T minus the row's previous element, RANGE the row's next element
-                            in[o + k] = Key<uint32_t>::make(T, OBJ == ZL_OBJ_SUM ? T - v[k] : k + 1 < c ? v[k + 2] : v[SUM_SHORT + 1]);
-                            rk[o + k] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
+                            in[o] = Key<uint32_t>::make(T, OBJ == ZL_OBJ_SUM ? T - v[k] : k + 1 < c ? v[k + 2] : v[SUM_SHORT + 1]);
+                            rk[o] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
                         }
                     }
                 } else {
-                    longs[atomicAdd(&sh.nlong, 1u)] = make_uint2((uint32_t)r | ((uint32_t)s << 16), (uint32_t)e | (o << 16));
+                    longs[atomicAdd(&sh.nlong, 1u)] = make_uint2((uint32_t)r | ((uint32_t)s << 16), (uint32_t)e | (o_run << 16));
                 }
             }
             myS = warp_reduce(myS, OpAdd());
             myC = warp_reduce(myC, OpAdd());
             if (lane == 0 && myC) { atomicAdd(&sh.carryS, (unsigned long long)myS); atomicAdd(&sh.carryC, myC); }
             __syncthreads();
-            const uint32_t m = sh.fill;
-            if (m > (uint32_t)cap) { over = true; break; }         // uniform over the block
+            if (OBJ == ZL_OBJ_SUM && sh.fill > (uint32_t)cap) { over = true; break; }   // uniform over the block
             const int nlong = (int)sh.nlong;
             uint64_t cS = sh.carryS;
             uint32_t cC = sh.carryC;
-            if (m == 0) continue;
+            if (OBJ == ZL_OBJ_SUM && sh.fill == 0) continue;
             for (int w = warp; w < nlong; w += nw) {
                 const uint2 d = longs[w];
                 const int r = (int)(d.x & 0xffffu), s = (int)(d.x >> 16), e = (int)(d.y & 0xffffu);
                 const uint32_t o = d.y >> 16;
                 const int64_t *rp = inst + (size_t)r * R;
-                for (int i = s + lane; i < e; i += 32) {
-                    const uint32_t T = (uint32_t)(uint64_t)ldg64(rp + i) - tminlo;
-                    uint32_t pay;
-                    if (OBJ == ZL_OBJ_SUM) pay = T - (i > 0 ? (uint32_t)(uint64_t)ldg64(rp + i - 1) - tminlo : 0u);
-                    else pay = i + 1 < R ? (uint32_t)(uint64_t)ldg64(rp + i + 1) - tminlo : 0xffffffffu;
-                    const uint32_t pos = o + (uint32_t)(i - s);
-                    in[pos] = Key<uint32_t>::make(T, pay);
-                    rk[pos] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
+                for (int i0 = s; i0 < e; i0 += 32) {
+                    const int i = i0 + lane;
+                    const uint32_t T = i < e ? (uint32_t)(uint64_t)ldg64(rp + i) - tminlo : 0xffffffffu;
+                    uint32_t pay, pos;
+                    if (OBJ == ZL_OBJ_SUM) {
+                        pay = T - (i > 0 && i < e ? (uint32_t)(uint64_t)ldg64(rp + i - 1) - tminlo : 0u);
+                        pos = o + (uint32_t)(i - s);
+                    } else {
+                        pay = i + 1 < R ? (uint32_t)(uint64_t)ldg64(rp + i + 1) - tminlo : 0xffffffffu;
+                        // the row is sorted: the lanes that stay are a prefix of the warp
+                        const unsigned keep = __ballot_sync(FULL, i < e && T <= tcut);
+                        unsigned base = 0;
+                        if (lane == 0 && keep) base = atomicAdd(&sh.fill, (unsigned)__popc(keep));
+                        pos = __shfl_sync(FULL, base, 0) + (uint32_t)lane;
+                        if (!((keep >> lane) & 1u)) pos = 0xffffffffu;
+                        if (keep != FULL) i0 = e;                 // the rest of the row lies after the cut (or the run ends)
+                    }
+                    if (i < e && pos < (uint32_t)cap) {
+                        in[pos] = Key<uint32_t>::make(T, pay);
+                        rk[pos] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
+                    }
                 }
             }
             __syncthreads();
+            const uint32_t m = sh.fill;
+            if (m > (uint32_t)cap) { over = true; break; }         // uniform over the block (cannot happen for a single bucket)
+            if (m == 0) continue;
             // slot counts -> slot starts
             uint32_t loc = 0, big = 0;
             for (int s = s0; s < s1; ++s) { const uint32_t c = cnt[slot_pad(s)]; loc += c; big |= c > (uint32_t)SLOT_MAX; }
@@ -1938,10 +1957,10 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         const size_t bsmem = (size_t)fb.scap * 18 + ((size_t)fb.scap + fb.scap / 32 + 2) * 4;
         if (q.objective == ZL_OBJ_SUM)
             launch_dep(!((q.pdl_off >> 3) & 1), zl::k_sum_buckets<ZL_OBJ_SUM>, dim3(std::min(items, 32 * q.num_sms)), dim3(bthreads), bsmem, st,
-                       q.ts, q.n, q.R, q.B, q.meta, fb, q.nres, q.seg);
+                       q.ts, q.n, q.R, q.B, 0, q.meta, fb, q.nres, q.seg);
         else
             launch_dep(!((q.pdl_off >> 3) & 1), zl::k_sum_buckets<ZL_OBJ_RANGE>, dim3(std::min(items, 32 * q.num_sms)), dim3(bthreads), bsmem, st,
-                       q.ts, q.n, q.R, q.B, q.meta, fb, q.nres, q.seg);
+                       q.ts, q.n, q.R, q.B, (q.flags & ZL_FLAG_FULL_SWEEP) ? 0 : 1, q.meta, fb, q.nres, q.seg);
     } else if (ev) {
         cudaEventRecord(ev[2], st);
     }
