@@ -244,7 +244,7 @@ zl_status zl_filter_counts(zl_handle *h, int32_t B, uint32_t *h_filtered, uint32
  * "segments" (time segments per instance, >= 1), "round_factor" (percent of the
  * nominal elements per round), "no_filter" (1: neither the RANGE filter route nor the bucket
  * route is used; every instance is swept by time segments), "filter_threads" / "filter_rows" (CTA size and rows per CTA of the
- * filter pass), "prologue_threads" / "tail_threads" (CTA sizes of those kernels), "pdl_off" (bit k: launch the k-th kernel of the chain only after its predecessor has
+ * filter pass), "filter_round" (a row is requested up to its estimate rounded up to this many timestamps; power of two, 2..256), "prologue_threads" / "tail_threads" (CTA sizes of those kernels), "pdl_off" (bit k: launch the k-th kernel of the chain only after its predecessor has
  * finished instead of scheduling it early).  0 restores the built-in choice. */
 zl_status zl_set_option(zl_handle *h, const char *key, int32_t value);
 

@@ -377,7 +377,7 @@ __device__ __forceinline__ uint32_t filter_slot_inside(const FilterCtx &C, const
     return __shfl_sync(FULL, b1, 31);
 }
 
-__global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R, int flags, int rows_per_cta,
+__global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R, int flags, int rows_per_cta, int req_round,
                                                   InstMeta *meta, FilterBufs F) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
@@ -408,7 +408,7 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
     for (int rbase = r0 + warp; rbase < r1; rbase += 32 * nw) {
         const int nrows = min(32, (r1 - rbase + nw - 1) / nw);
         int req = 0;
-        if (lane < nrows) req = full ? R : min(R, (int)((F.rowhint[(size_t)b * n + rbase + lane * nw] + 63) & ~63u));
+        if (lane < nrows) req = full ? R : min(R, (int)((F.rowhint[(size_t)b * n + rbase + lane * nw] + (uint32_t)(req_round - 1)) & ~(uint32_t)(req_round - 1)));
         const int64_t *row_i = ts + ((size_t)b * n + rbase) * R, *row_p = row_i;
         int ji = 0, ci = 0, jp = 0, cp = 0, inflight = 0, slot_i = 0, slot_p = 0;
         int req_i = __shfl_sync(FULL, req, 0), req_p = req_i;
@@ -1852,7 +1852,7 @@ struct zl_handle {
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round;
     int last_cuda_error;
     int launches;
     // optional per-kernel timing: PROF_EVENTS events per recorded call
@@ -1873,7 +1873,7 @@ struct Pipeline {
     const int64_t *ts; int B, n, R, objective, flags, num_sms;
     zl::InstMeta *meta; zl::SegResult *seg; int nres;
     zl::FilterBufs fb;                                            // fb.table == nullptr: no filter route
-    int filter_threads, filter_rows;                              // 0: automatic
+    int filter_threads, filter_rows, filter_round;                // 0: automatic
     int pdl_off;                                                  // bit mask of kernels launched without early scheduling
     int prologue_threads, tail_threads;                           // 0: automatic
     int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;
@@ -1922,7 +1922,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         fb.nreg = (int)((q.n + rpc - 1) / rpc);
         fb.regcap = fb.list1cap / fb.nreg;
         const size_t fsmem = (size_t)fb.cells * 4 + (size_t)nw * zl::FILTER_STAGES * zl::FILTER_SLOT * 8;
-        launch_dep(!((q.pdl_off >> 1) & 1), zl::k_filter, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.flags, (int)rpc, q.meta, fb);
+        launch_dep(!((q.pdl_off >> 1) & 1), zl::k_filter, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.flags, (int)rpc, q.filter_round ? q.filter_round : 8, q.meta, fb);
         if (ev) cudaEventRecord(ev[2], st);
         const int tcap = (int)std::min<long long>((long long)zl::TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
         launch_dep(!((q.pdl_off >> 2) & 1), zl::k_tail, dim3(q.B), dim3(q.tail_threads ? q.tail_threads : many ? (tcap <= 1024 ? 128 : 256) : std::max(64, std::min(1024, tcap / 2))), (size_t)tcap * 20 + (size_t)fb.cells * 4, st,
@@ -2227,6 +2227,9 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
         (key[0] == 'p' ? h->opt_prologue_threads : h->opt_tail_threads) = value;
     } else if (!strcmp(key, "pdl_off")) {
         h->opt_pdl_off = value;                 // bit k set: kernel k of the chain is launched without early scheduling
+    } else if (!strcmp(key, "filter_round")) {
+        if (value && (!is_pow2(value) || value < 2 || value > 256)) return ZL_ERR_INVALID_ARG;
+        h->opt_filter_round = value;
     } else if (!strcmp(key, "filter_rows")) {
         if (value > 65536) return ZL_ERR_INVALID_ARG;
         h->opt_filter_rows = value;
@@ -2271,7 +2274,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.ts = d_ts; q.B = B; q.n = n; q.R = R; q.objective = obj; q.flags = h->cfg.flags; q.num_sms = h->num_sms;
     q.meta = h->d_meta; q.seg = h->d_seg; q.nres = h->nres;
     q.fb = h->fb;
-    q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.pdl_off = h->opt_pdl_off;
+    q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.filter_round = h->opt_filter_round; q.pdl_off = h->opt_pdl_off;
     q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
     if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
@@ -2447,7 +2450,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
     q.meta = meta; q.seg = seg; q.nres = p.nseg;
     memset(&q.fb, 0, sizeof(q.fb));
-    q.filter_threads = q.filter_rows = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0;
+    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr);
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;

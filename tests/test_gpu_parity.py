@@ -118,7 +118,8 @@ def test_launch_shapes_do_not_change_results(objective):
     ref = gpu_select(ts, objective)
     assert_same(ts, objective, ref)
     for opts in ({"segments": 7}, {"segments": 16, "threads": 128}, {"lanes_per_row": 1, "threads": 256},
-                 {"lanes_per_row": 32, "segments": 3}, {"round_factor": 5}, {"round_factor": 2000, "segments": 2}):
+                 {"lanes_per_row": 32, "segments": 3}, {"round_factor": 5}, {"round_factor": 2000, "segments": 2},
+                 {"filter_round": 2}, {"filter_round": 8, "filter_threads": 64}, {"filter_round": 256}):
         got = gpu_select(ts, objective, options=opts)
         for a, b in zip(ref, got):
             assert (a == b).all(), opts
