@@ -154,10 +154,14 @@ __global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, 
     __shared__ uint64_t s[4][32];
     __shared__ InstMeta sm;
     __shared__ uint32_t tab[FILTER_MAX_CELLS];
+    extern __shared__ __align__(16) unsigned char smem[];
+    int64_t *col1 = (int64_t *)smem, *colR = col1 + n;        // first and last column: read once, used three times
     uint64_t mn1 = ~0ull, mx1 = 0, mnR = ~0ull, mxR = 0;      // order-preserving unsigned images of int64
     for (int p = tid; p < n; p += nt) {
-        const uint64_t e1 = (uint64_t)ldg64(inst + (size_t)p * R) ^ (1ull << 63);
-        const uint64_t eR = (uint64_t)ldg64(inst + (size_t)p * R + R - 1) ^ (1ull << 63);
+        const int64_t r1 = ldg64(inst + (size_t)p * R), rR = ldg64(inst + (size_t)p * R + R - 1);
+        col1[p] = r1; colR[p] = rR;
+        const uint64_t e1 = (uint64_t)r1 ^ (1ull << 63);
+        const uint64_t eR = (uint64_t)rR ^ (1ull << 63);
         mn1 = min(mn1, e1); mx1 = max(mx1, e1);
         mnR = min(mnR, eR); mxR = max(mxR, eR);
     }
@@ -205,8 +209,8 @@ __global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, 
         // per row: how many of its elements are expected to be <= lmin (rows are close to arithmetic);
         // the filter pass uses it only to decide how much of the row to request up front
         for (int p = tid; p < n; p += nt) {
-            const uint64_t e1 = (uint64_t)(ldg64(inst + (size_t)p * R) - tmin) + 1;
-            const uint64_t eR = (uint64_t)(ldg64(inst + (size_t)p * R + R - 1) - tmin) + 1;
+            const uint64_t e1 = (uint64_t)(col1[p] - tmin) + 1;
+            const uint64_t eR = (uint64_t)(colR[p] - tmin) + 1;
             uint64_t est = R;
             if (eR > e1 && (uint64_t)lmin < eR)
                 est = (uint64_t)lmin <= e1 ? 1 : ((uint64_t)lmin - e1) * (uint64_t)(R - 1) / (eR - e1) + 8;
@@ -221,7 +225,7 @@ __global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, 
             int bestp = -1;
             uint64_t bspan = 0;
             for (int p = p0 + lane; p < p1; p += 32) {
-                const uint64_t span = (uint64_t)(ldg64(inst + (size_t)p * R + R - 1) - ldg64(inst + (size_t)p * R));
+                const uint64_t span = (uint64_t)(colR[p] - col1[p]);
                 if (bestp < 0 || span > bspan) { bspan = span; bestp = p; }
             }
             const uint64_t best = warp_reduce(bspan, OpMax());
@@ -1905,7 +1909,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     const bool many = q.B > 2 * q.num_sms;
     const int pthreads = q.prologue_threads ? q.prologue_threads
                          : many ? std::max(128, std::min(256, pow2_ceil(2 * q.n))) : std::max(512, std::min(1024, pow2_ceil(q.n)));
-    zl::k_prologue<<<q.B, pthreads, 0, st>>>(q.ts, q.n, q.R, q.objective, q.flags, q.meta, fb);
+    zl::k_prologue<<<q.B, pthreads, (size_t)q.n * 16, st>>>(q.ts, q.n, q.R, q.objective, q.flags, q.meta, fb);
     if (q.flags & ZL_FLAG_CHECK_SORTED) {
         const size_t total = (size_t)q.B * q.n * q.R;
         const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)q.num_sms * 16);
@@ -1988,6 +1992,7 @@ cudaError_t raise_shared_memory_limits() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_buckets, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_tail, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_prologue, cudaFuncAttributeMaxDynamicSharedMemorySize, zl::MAX_WORKERS * 16);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_buckets<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_buckets<ZL_OBJ_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_plan, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
