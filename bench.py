@@ -268,6 +268,38 @@ def main():
     hf.destroy()
     clocks = sampler.stop()
 
+    # what the memory system delivers for the bytes of the filter pass: a kernel that only loads them (a warp per row, the
+    # row prefixes the early stop needs, then whole rows), with the L2 flushed before each launch and as run back to back
+    probe = None
+    if rank == 0 and h.route == 1:
+        lmin_row = ts_np[:, :, -1].min(axis=1)
+        cnt = (ts_np <= lmin_row[:, None, None]).sum(axis=2).astype(np.int64)
+        pref = np.minimum(w.R, (cnt + 8 + 7) // 8 * 8).astype(np.int32).reshape(-1)     # as the filter pass requests them
+        d_pref = torch.from_numpy(pref).to(dev)
+        d_full = torch.full_like(d_pref, w.R)
+        sink = torch.zeros(1, dtype=torch.int64, device=dev)
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+        def probe_us(counts, cold, reps=10):
+            tot = 0.0
+            for i in range(reps + 2):
+                if cold:
+                    flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                zl.zl_probe_read_batched(d_ts[i % copies], counts, sink)
+                b.record()
+                torch.cuda.synchronize()
+                if i >= 2:
+                    tot += a.elapsed_time(b)
+            return tot / reps * 1e3
+        probe = {"prefix_bytes": int(pref.astype(np.int64).sum()) * 8,
+                 "prefix_us_cold_l2": probe_us(d_pref, True), "prefix_us": probe_us(d_pref, False),
+                 "full_bytes": nts * 8, "full_us_cold_l2": probe_us(d_full, True), "full_us": probe_us(d_full, False),
+                 "what": "load-only kernel on the bytes of the filter pass (row prefixes up to the first exhausted row, "
+                         "then whole rows); cold = 256 MB written before each launch"}
+        del flush
+
     # end to end: host buffers in, host results out, through the C ABI
     e2e_steps = max(3, min(args.steps, 10))
     ms_e, _, _ = timed(h, e2e_steps, 3, host=True)
@@ -330,7 +362,8 @@ def main():
             "vs_baseline": None, "dtype": "int64", "data": "synthetic", "config": cfg, "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "timestamps/s", "h2d_bytes_per_step": nts * 8,
                     "d2h_bytes_per_step": w.B * (4 * w.n + 20), "ms_per_step": ms_e / e2e_steps},
-            "gpu_launches": launches, "roofline": roofline, "full_sweep": full, "cpu_baseline": cpu}
+            "gpu_launches": launches, "roofline": roofline, "full_sweep": full, "cpu_baseline": cpu,
+            "load_only_probe": probe}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

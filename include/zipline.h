@@ -225,6 +225,21 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
 int32_t  zl_noalloc_max_batch(void);       /* largest B of zl_select_batched_noalloc           */
 size_t   zl_noalloc_scratch_bytes(void);   /* size of the fixed device array it works in       */
 
+/*
+ * Measurement aid (no counterpart in the paper): a kernel that only loads, a warp per row, the first
+ * d_count[row] timestamps of each of `rows` rows of length R (16-byte loads where the layout allows)
+ * and does nothing else.  bench.py times it on the bytes the filter pass of the search reads, to show what
+ * the memory system delivers for that access pattern.
+ *
+ *   d_ts     device, [rows][R] int64, 8-byte aligned.
+ *   d_count  device, [rows] int32: how many leading timestamps of the row to read (clamped to 0..R).
+ *   d_sink   device, one uint64 the caller owns (receives a checksum practically never; keeps the loads alive).
+ *
+ * Asynchronous on cuda_stream; no handle, no scratch, no allocation.
+ */
+zl_status zl_probe_read_batched(const int64_t *d_ts, const int32_t *d_count, int64_t rows, int32_t R,
+                                uint64_t *d_sink, void *cuda_stream);
+
 /* Free the scratch and the handle.  NULL is a no-op. */
 zl_status zl_destroy(zl_handle *h);
 

@@ -23,7 +23,8 @@ EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace
            "zl_segments_per_instance", "zl_max_workers", "zl_trace_max_elements", "zl_last_cuda_error",
            "zl_profile_begin", "zl_profile_read", "zl_profile_end",
            "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes", "zl_filter_counts",
-           "zl_predict_batched", "zl_predict_select_batched", "zl_gridscan_batched", "zl_route")
+           "zl_predict_batched", "zl_predict_select_batched", "zl_gridscan_batched", "zl_route",
+           "zl_probe_read_batched")
 
 
 class zl_config(ctypes.Structure):
@@ -47,6 +48,8 @@ def _load() -> ctypes.CDLL:
     lib.zl_launches_per_call.argtypes = [vp]
     lib.zl_segments_per_instance.argtypes = [vp, i32]
     lib.zl_route.argtypes = [vp]
+    lib.zl_probe_read_batched.argtypes = [vp, vp, ctypes.c_int64, i32, vp, vp]
+    lib.zl_probe_read_batched.restype = ctypes.c_int
     lib.zl_route.restype = ctypes.c_int
     lib.zl_last_cuda_error.argtypes = [vp]
     lib.zl_profile_begin.argtypes = [vp, i32]
@@ -264,6 +267,18 @@ def zl_gridscan_batched(ts: torch.Tensor, full: bool = False, stream: torch.cuda
                                  scratch.data_ptr(), idx.data_ptr(), barrier.data_ptr(), wait.data_ptr(), s.cuda_stream)
     _check(rc, "zl_gridscan_batched")
     return idx, barrier, wait
+
+
+def zl_probe_read_batched(ts: torch.Tensor, count: torch.Tensor, sink: torch.Tensor,
+                          stream: torch.cuda.Stream | None = None) -> None:
+    """Measurement aid: only load the first count[row] timestamps of every row.
+    ts: CUDA int64 [..., R]; count: CUDA int32, one per row; sink: CUDA int64/uint64 scalar."""
+    R = ts.shape[-1]
+    rows = ts.numel() // R
+    s = stream if stream is not None else torch.cuda.current_stream(ts.device)
+    rc = lib.zl_probe_read_batched(_dev_ptr(ts, torch.int64, rows * R, "ts"), _dev_ptr(count, torch.int32, rows, "count"),
+                                   rows, R, sink.data_ptr(), s.cuda_stream)
+    _check(rc, "zl_probe_read_batched")
 
 
 def zl_noalloc_max_batch() -> int:

@@ -221,6 +221,19 @@ def test_host_buffer_entry_point_and_streams():
     h.destroy()
 
 
+def test_read_probe_runs_on_any_layout():
+    # the load-only measurement kernel: even and odd row lengths, counts beyond the row are clamped
+    for R in (64, 77, 1024):
+        ts = torch.arange(40 * R, dtype=torch.int64, device="cuda").reshape(40, R)
+        count = torch.tensor([0, 1, R - 1, R, R + 50] * 8, dtype=torch.int32, device="cuda")
+        sink = torch.zeros(1, dtype=torch.int64, device="cuda")
+        zl.zl_probe_read_batched(ts, count, sink)
+        zl.zl_probe_read_batched(ts[1:, :], count[1:], sink)           # rows that start 8 bytes off a 16-byte boundary when R is odd
+        torch.cuda.synchronize()
+    with pytest.raises(ValueError):
+        zl.zl_probe_read_batched(ts, count[:3], sink)
+
+
 # ---------------------------------------------------------------- per-step intermediates
 def test_trace_matches_oracle_trace():
     rng = np.random.default_rng(17)
