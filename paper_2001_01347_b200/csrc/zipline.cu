@@ -1351,14 +1351,21 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
                 const int r = (int)(d.x & 0xffffu), s = (int)(d.x >> 16), e = (int)(d.y & 0xffffu);
                 const uint32_t o = d.y >> 16;
                 const int64_t *rp = inst + (size_t)r * R;
+                if (OBJ == ZL_OBJ_SUM) {
+                    for (int i = s + lane; i < e; i += 32) {
+                        const uint32_t T = (uint32_t)(uint64_t)ldg64(rp + i) - tminlo;
+                        const uint32_t pv = i > 0 ? (uint32_t)(uint64_t)ldg64(rp + i - 1) - tminlo : 0u;
+                        const uint32_t pos = o + (uint32_t)(i - s);
+                        in[pos] = Key<uint32_t>::make(T, T - pv);
+                        rk[pos] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
+                    }
+                    continue;
+                }
                 for (int i0 = s; i0 < e; i0 += 32) {
                     const int i = i0 + lane;
                     const uint32_t T = i < e ? (uint32_t)(uint64_t)ldg64(rp + i) - tminlo : 0xffffffffu;
                     uint32_t pay, pos;
-                    if (OBJ == ZL_OBJ_SUM) {
-                        pay = T - (i > 0 && i < e ? (uint32_t)(uint64_t)ldg64(rp + i - 1) - tminlo : 0u);
-                        pos = o + (uint32_t)(i - s);
-                    } else {
+                    {
                         pay = i + 1 < R ? (uint32_t)(uint64_t)ldg64(rp + i + 1) - tminlo : 0xffffffffu;
                         // the row is sorted: the lanes that stay are a prefix of the warp
                         const unsigned keep = __ballot_sync(FULL, i < e && T <= tcut);
