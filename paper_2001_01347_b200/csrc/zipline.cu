@@ -1951,7 +1951,8 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     const bool many = q.B > 2 * q.num_sms;
     const int pthreads = q.prologue_threads ? q.prologue_threads
                          : many ? std::max(128, std::min(256, pow2_ceil(2 * q.n))) : std::max(512, std::min(1024, pow2_ceil(q.n)));
-    zl::k_prologue<<<q.B, pthreads, (size_t)q.n * 16, st>>>(q.ts, q.n, q.R, q.objective, q.flags, q.meta, fb);
+    // the first kernel of a call is scheduled early too: it waits (grid_dep_wait) for whatever precedes it in the stream
+    launch_dep(!((q.pdl_off >> 9) & 1), zl::k_prologue, dim3(q.B), dim3(pthreads), (size_t)q.n * 16, st, q.ts, q.n, q.R, q.objective, q.flags, q.meta, fb);
     if (q.flags & ZL_FLAG_CHECK_SORTED) {
         const size_t total = (size_t)q.B * q.n * q.R;
         const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)q.num_sms * 16);
