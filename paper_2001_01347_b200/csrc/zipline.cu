@@ -43,6 +43,7 @@
 #include <algorithm>
 #include <mutex>
 #include <new>
+#include <type_traits>
 
 #include "../../include/zipline.h"
 #include "zl_device.cuh"
@@ -75,6 +76,43 @@ struct SegResult {
     uint64_t t;          // its relative time (min(Z) for RANGE, the barrier for SUM)
     int32_t valid;
     int32_t status;
+};
+
+// Where the rows of an instance come from: the stored [B][n][R] matrix, or - for predicted rows - the
+// rule e_i = last + (i + 1) * interval itself, so that the matrix never has to exist in memory.  A worker with
+// a negative input reads as a row of -1, one whose last prediction would reach 2^62 as a row of 2^62: both
+// make the column scans report the instance invalid.
+struct MatRow {
+    const int64_t *p;
+    __device__ __forceinline__ int64_t at(int i) const { return (int64_t)__ldg((const long long *)(p + i)); }
+};
+struct AriRow {
+    int64_t l, v;
+    __device__ __forceinline__ int64_t at(int i) const { return l + (int64_t)(i + 1) * v; }
+};
+struct MatRows {
+    const int64_t *inst; int R;
+    __device__ __forceinline__ MatRow row(int p) const { return MatRow{inst + (size_t)p * R}; }
+};
+struct AriRows {
+    const int64_t *last, *iv; int R;
+    __device__ __forceinline__ AriRow row(int p) const {
+        const int64_t l = (int64_t)__ldg((const long long *)(last + p)), v = (int64_t)__ldg((const long long *)(iv + p));
+        if (l < 0 || v < 0) return AriRow{-1, 0};
+        if (__umul64hi((uint64_t)R, (uint64_t)v) != 0 || (uint64_t)R * (uint64_t)v >= (uint64_t)VALUE_LIMIT ||
+            (uint64_t)l + (uint64_t)R * (uint64_t)v >= (uint64_t)VALUE_LIMIT) return AriRow{VALUE_LIMIT, 0};
+        return AriRow{l, v};
+    }
+};
+struct MatBatch {
+    const int64_t *ts;
+    typedef MatRows Rows;
+    __device__ __forceinline__ MatRows inst(int b, int n, int R) const { return MatRows{ts + (size_t)b * n * R, R}; }
+};
+struct AriBatch {
+    const int64_t *last, *iv;
+    typedef AriRows Rows;
+    __device__ __forceinline__ AriRows inst(int b, int n, int R) const { return AriRows{last + (size_t)b * n, iv + (size_t)b * n, R}; }
 };
 
 // Buffers of the RANGE filter route (all nullptr / 0 when the route is off).  The time up to lmin is
@@ -146,11 +184,12 @@ __device__ __forceinline__ bool tail_instance(const InstMeta &M) { return M.coun
 constexpr int FILTER_ROWS = 32;      // rows that build the table
 constexpr int FILTER_MAX_CELLS = 8192;
 
-__global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, int R, int objective, int flags,
+template <class SRC>
+__global__ void __launch_bounds__(1024, 1) k_prologue(const SRC src, int n, int R, int objective, int flags,
                                                     InstMeta *meta, FilterBufs F) {
     grid_dep_wait();
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
-    const int64_t *inst = ts + (size_t)b * n * R;
+    const typename SRC::Rows rows = src.inst(b, n, R);
     __shared__ uint64_t s[4][32];
     __shared__ InstMeta sm;
     __shared__ uint32_t tab[FILTER_MAX_CELLS];
@@ -158,7 +197,8 @@ __global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, 
     int64_t *col1 = (int64_t *)smem, *colR = col1 + n;        // first and last column: read once, used three times
     uint64_t mn1 = ~0ull, mx1 = 0, mnR = ~0ull, mxR = 0;      // order-preserving unsigned images of int64
     for (int p = tid; p < n; p += nt) {
-        const int64_t r1 = ldg64(inst + (size_t)p * R), rR = ldg64(inst + (size_t)p * R + R - 1);
+        const auto rw = rows.row(p);
+        const int64_t r1 = rw.at(0), rR = rw.at(R - 1);
         col1[p] = r1; colR[p] = rR;
         const uint64_t e1 = (uint64_t)r1 ^ (1ull << 63);
         const uint64_t eR = (uint64_t)rR ^ (1ull << 63);
@@ -232,7 +272,7 @@ __global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, 
             const unsigned who = __ballot_sync(FULL, bestp >= 0 && bspan == best);
             if (!who) continue;
             const int row = __shfl_sync(FULL, bestp, __ffs(who) - 1);
-            const int64_t *rp = inst + (size_t)row * R;
+            const auto rp = rows.row(row);
             // element i is the first element of the row at or after every cell start in (e_{i-1}, e_i]:
             // the cells after the one holding e_{i-1}, up to the one holding e_i
             // (four 32-element steps are loaded before any is used: the loop is latency bound otherwise)
@@ -243,8 +283,8 @@ __global__ void __launch_bounds__(1024, 1) k_prologue(const int64_t *ts, int n, 
                     const int i = i0 + 32 * k + lane;
                     pv[k] = 0xffffffffu; cv[k] = 0;
                     if (i < R) {
-                        pv[k] = (uint32_t)(ldg64(rp + i - 1) - tmin + 1);
-                        cv[k] = (uint32_t)(ldg64(rp + i) - tmin + 1);
+                        pv[k] = (uint32_t)(rp.at(i - 1) - tmin + 1);
+                        cv[k] = (uint32_t)(rp.at(i) - tmin + 1);
                     }
                 }
 #pragma unroll
@@ -498,6 +538,56 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
     }
 }
 
+// The filter pass on predicted rows e_i = last + (i + 1) * interval, which are generated instead of read.  An
+// element's own iteration is the row's interval, so a whole row whose interval does not exceed dmin is settled
+// at once (only its last element, whose next is infinite, can pass); the other rows are walked up to lmin, an
+// element per lane.  Same regions, lists and counters as k_filter.
+__global__ void __launch_bounds__(256) k_filter_arith(const AriBatch src, int n, int R, int rows_per_cta, InstMeta *meta, FilterBufs F) {
+    grid_dep_wait();
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ unsigned int scount;
+    const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+    const InstMeta M = meta[b];
+    uint32_t *rc = F.rcnt + (size_t)b * F.nreg + blockIdx.x;
+    if (M.status != ZL_OK || M.cscale == 0) { if (tid == 0) *rc = 0; return; }
+    const uint32_t cells = (uint32_t)F.cells;
+    uint32_t *tab = (uint32_t *)smem;
+    const uint32_t *tg = F.table + (size_t)b * cells;
+    for (uint32_t c = tid; c < cells; c += nt) tab[c] = tg[c];
+    if (tid == 0) scount = 0;
+    __syncthreads();
+    FilterCtx C;
+    C.tab = tab; C.list = F.list1 + (size_t)b * F.list1cap + (size_t)blockIdx.x * F.regcap;
+    C.cellmax = F.cellmax + (size_t)b * F.fcells; C.scount = &scount;
+    C.cscale = M.cscale; C.fscale = M.fscale; C.lmin = (uint32_t)M.lmin; C.regcap = (uint32_t)F.regcap; C.dmin = M.dmin;
+    const AriRows rows = src.inst(b, n, R);
+    const int r0 = blockIdx.x * rows_per_cta, r1 = min(r0 + rows_per_cta, n);
+    for (int r = r0 + warp; r < r1; r += nw) {
+        const AriRow rw = rows.row(r);
+        const int64_t rel0 = rw.l - M.tmin + 1;                   // relative time of element i: rel0 + (i + 1) * v, >= 1
+        const int64_t v = rw.v, room = (int64_t)M.lmin - rel0;
+        // elements not after lmin: (i + 1) * v <= room
+        const int cnt = v == 0 ? (room >= 0 ? R : 0) : room < v ? 0 : (int)min((int64_t)R, room / v);
+        if (cnt == 0) continue;
+        if ((uint64_t)v <= (uint64_t)M.dmin) {
+            if (cnt == R) filter_pair(C, lane, lane == 0, (uint32_t)(rel0 + (int64_t)R * v), 0xffffffffu, false, 0u, 0u);
+            continue;
+        }
+        for (int i0 = 0; i0 < cnt; i0 += 32) {
+            const int i = i0 + lane;
+            const uint32_t T = (uint32_t)(rel0 + (int64_t)(i + 1) * v);
+            filter_pair(C, lane, i < cnt, T, i + 1 < R ? T + (uint32_t)v : 0xffffffffu, false, 0u, 0u);
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned c = scount;
+        *rc = min(c, (unsigned)F.regcap);
+        if (c > (unsigned)F.regcap) meta[b].overflow = 1;
+        if (c) atomicAdd(&meta[b].count, c);
+    }
+}
+
 // ------------------------------------------------------------------------------ refinement (RANGE)
 // The per-cell maxima of the filter pass give G exactly at every fine cell start (the survivors contain
 // every element that ever raises the running maximum): k_cellscan turns cellmax, in place, into its
@@ -734,8 +824,8 @@ struct SweepShared {
     uint64_t tmp[34];
 };
 
-template <typename K, int OBJ>
-__device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int64_t *inst, SweepShared &sh,
+template <typename K, int OBJ, class ROWS>
+__device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const ROWS &rows, SweepShared &sh,
                               uint32_t *curA, uint32_t *curB, const BatchWS<K> &ws, int seg_index, SegResult &out) {
     Key<K> *keys = ws.in;
     const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
@@ -768,19 +858,19 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
             unsigned long long vloc = 0, sloc = 0;
             unsigned int cloc = 0;
             for (int r = tid; r < n; r += nt) {
-                const int64_t *row = inst + (size_t)r * R;
+                const auto row = rows.row(r);
                 int lo = 0, hi = R;               // first index with row[i] >= a_raw
                 while (lo < hi) {
                     const int mid = (lo + hi) >> 1;
-                    if (ldg64(row + mid) < a_raw) lo = mid + 1; else hi = mid;
+                    if (row.at(mid) < a_raw) lo = mid + 1; else hi = mid;
                 }
                 curA[r] = (uint32_t)lo;
                 if (lo > 0) {
                     if (OBJ == ZL_OBJ_RANGE) {
-                        const unsigned long long v = lo < R ? (unsigned long long)(K)(ldg64(row + lo) - tmin + 1) : (unsigned long long)INF;
+                        const unsigned long long v = lo < R ? (unsigned long long)(K)(row.at(lo) - tmin + 1) : (unsigned long long)INF;
                         vloc = max(vloc, v);
                     } else {
-                        sloc += (unsigned long long)(K)(ldg64(row + lo - 1) - tmin + 1);
+                        sloc += (unsigned long long)(K)(row.at(lo - 1) - tmin + 1);
                         cloc += 1;
                     }
                 }
@@ -822,25 +912,25 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
             for (int rb = 0; rb < n; rb += NG) {
                 const int r = rb + gi;
                 const bool act = r < n;
-                const int64_t *row = inst + (size_t)(act ? r : 0) * R;
+                const auto row = rows.row(act ? r : 0);
                 uint32_t c = act ? cur[r] : (uint32_t)R;
                 bool more = act;
                 for (;;) {
                     const uint32_t idx = c + g;
                     const bool have = more && idx < (uint32_t)R;
-                    const K T = have ? (K)(ldg64(row + idx) - tmin + 1) : INF;
+                    const K T = have ? (K)(row.at((int)idx) - tmin + 1) : INF;
                     const bool cons = have && T < rhi;
                     bool app = false;
                     Key<K> key = Key<K>::inf();
                     if (cons) {
                         ++cons_n;
                         if (OBJ == ZL_OBJ_RANGE) {
-                            const K nx = idx + 1 < (uint32_t)R ? (K)(ldg64(row + idx + 1) - tmin + 1) : INF;
+                            const K nx = idx + 1 < (uint32_t)R ? (K)(row.at((int)idx + 1) - tmin + 1) : INF;
                             vloc = max(vloc, (unsigned long long)nx);
                             app = nx > max(T, floorv);            // only elements that raise the running max matter
                             key = Key<K>::make(T, nx);
                         } else {
-                            const K pv = idx > 0 ? (K)(ldg64(row + idx - 1) - tmin + 1) : (K)0;
+                            const K pv = idx > 0 ? (K)(row.at((int)idx - 1) - tmin + 1) : (K)0;
                             app = idx == 0 || T != pv;             // repeated timestamps of a row add nothing
                             key = Key<K>::make(T, T - pv);
                         }
@@ -919,8 +1009,8 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const int
     block_best_to_result(bd, bt, status, sh.tmp, &sh.status, out);
 }
 
-template <int OBJ>
-__global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
+template <int OBJ, class SRC>
+__global__ void __launch_bounds__(1024) k_sweep(const SweepParams P, const SRC src) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ SweepShared sh;
@@ -942,7 +1032,7 @@ __global__ void __launch_bounds__(1024) k_sweep(const SweepParams P) {
             if (threadIdx.x == 0) { out.d = ~0ull; out.t = ~0ull; out.valid = 0; out.status = ZL_OK; }
             continue;
         }
-        const int64_t *inst = P.ts + (size_t)b * P.n * P.R;
+        const typename SRC::Rows inst = src.inst(b, P.n, P.R);
         if (M.use32) {
             const BatchWS<uint32_t> ws{(Key<uint32_t> *)kb, (Key<uint32_t> *)kb2, kcnt, P.cap};
             sweep_segment<uint32_t, OBJ>(P, M, inst, sh, curA, curB, ws, sidx, out);
@@ -1359,25 +1449,21 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
                         in[pos] = Key<uint32_t>::make(T, T - pv);
                         rk[pos] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
                     }
-                    continue;
-                }
-                for (int i0 = s; i0 < e; i0 += 32) {
-                    const int i = i0 + lane;
-                    const uint32_t T = i < e ? (uint32_t)(uint64_t)ldg64(rp + i) - tminlo : 0xffffffffu;
-                    uint32_t pay, pos;
-                    {
-                        pay = i + 1 < R ? (uint32_t)(uint64_t)ldg64(rp + i + 1) - tminlo : 0xffffffffu;
+                } else {
+                    for (int i0 = s; i0 < e; i0 += 32) {
+                        const int i = i0 + lane;
+                        const uint32_t T = i < e ? (uint32_t)(uint64_t)ldg64(rp + i) - tminlo : 0xffffffffu;
+                        const uint32_t pay = i + 1 < R ? (uint32_t)(uint64_t)ldg64(rp + i + 1) - tminlo : 0xffffffffu;
                         // the row is sorted: the lanes that stay are a prefix of the warp
                         const unsigned keep = __ballot_sync(FULL, i < e && T <= tcut);
                         unsigned base = 0;
                         if (lane == 0 && keep) base = atomicAdd(&sh.fill, (unsigned)__popc(keep));
-                        pos = __shfl_sync(FULL, base, 0) + (uint32_t)lane;
-                        if (!((keep >> lane) & 1u)) pos = 0xffffffffu;
-                        if (keep != FULL) i0 = e;                 // the rest of the row lies after the cut (or the run ends)
-                    }
-                    if (i < e && pos < (uint32_t)cap) {
-                        in[pos] = Key<uint32_t>::make(T, pay);
-                        rk[pos] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
+                        const uint32_t pos = __shfl_sync(FULL, base, 0) + (uint32_t)lane;
+                        if (((keep >> lane) & 1u) && pos < (uint32_t)cap) {
+                            in[pos] = Key<uint32_t>::make(T, pay);
+                            rk[pos] = (uint16_t)atomicAdd(&cnt[slot_pad((int)min(__umulhi(T - lo, scale), (uint32_t)nslots - 1u))], 1u);
+                        }
+                        if (keep != FULL) break;                  // the rest of the row lies after the cut (or the run ends)
                     }
                 }
             }
@@ -1464,8 +1550,9 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
 // position is first guessed from the row's end points.  Eight probes around the guess, eight elements apart and
 // loaded together, then the seven elements between the two probes that bracket bar, loaded together: three
 // rounds of loads in the usual case.  A guess that is further off is bracketed by doubling steps and bisected.
-__device__ int last_index_not_after(const int64_t *row, int R, int64_t bar) {
-    const int64_t e0 = ldg64(row), eR = ldg64(row + R - 1);
+template <class ROW>
+__device__ int last_index_not_after(const ROW &row, int R, int64_t bar) {
+    const int64_t e0 = row.at(0), eR = row.at(R - 1);
     if (bar < e0) return -1;
     if (bar >= eR) return R - 1;
     // e0 <= bar < eR, R >= 2.  Invariant: row[lo - 1] <= bar, row[hi] > bar
@@ -1477,7 +1564,7 @@ __device__ int last_index_not_after(const int64_t *row, int R, int64_t bar) {
         int64_t pv[P];
         int pi[P];
 #pragma unroll
-        for (int k = 0; k < P; ++k) { pi[k] = max(0, min(R - 1, g + S * (k - P / 2))); pv[k] = ldg64(row + pi[k]); }
+        for (int k = 0; k < P; ++k) { pi[k] = max(0, min(R - 1, g + S * (k - P / 2))); pv[k] = row.at(pi[k]); }
         lo = 1; hi = R - 1;
 #pragma unroll
         for (int k = 0; k < P; ++k) {
@@ -1486,7 +1573,7 @@ __device__ int last_index_not_after(const int64_t *row, int R, int64_t bar) {
         if (hi - lo <= S - 1) {                            // bracketed between two neighbouring probes
             int64_t wv[S - 1];
 #pragma unroll
-            for (int k = 0; k < S - 1; ++k) wv[k] = ldg64(row + min(lo + k, R - 1));
+            for (int k = 0; k < S - 1; ++k) wv[k] = row.at(min(lo + k, R - 1));
             int c = 0;
 #pragma unroll
             for (int k = 0; k < S - 1; ++k) c += (lo + k < hi && wv[k] <= bar) ? 1 : 0;   // sorted: a prefix of the window
@@ -1499,17 +1586,17 @@ __device__ int last_index_not_after(const int64_t *row, int R, int64_t bar) {
         for (int step = 16; lo < hi; step <<= 1) {
             const int q = min(lo + step - 1, top - 1);
             if (q < lo) break;
-            if (ldg64(row + q) <= bar) lo = q + 1; else { hi = q; break; }
+            if (row.at(q) <= bar) lo = q + 1; else { hi = q; break; }
         }
     } else {                                               // everything probed was > bar: search downwards from hi
         for (int step = 16; lo < hi; step <<= 1) {
             const int q = max(hi - step, lo);
-            if (ldg64(row + q) > bar) hi = q; else { lo = q + 1; break; }
+            if (row.at(q) > bar) hi = q; else { lo = q + 1; break; }
         }
     }
     while (lo < hi) {
         const int mid = (lo + hi) >> 1;
-        if (ldg64(row + mid) <= bar) lo = mid + 1; else hi = mid;
+        if (row.at(mid) <= bar) lo = mid + 1; else hi = mid;
     }
     return lo - 1;
 }
@@ -1519,8 +1606,9 @@ __device__ int last_index_not_after(const int64_t *row, int R, int64_t bar) {
 // exclusive prefix maximum, drop every survivor whose next does not exceed the value at its cell's
 // start), then sorts what is left and sweeps it.  Dropped survivors never hold the running maximum
 // alone, so nothing has to be carried in.
+template <class SRC>
 __global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg, int tcap,
-                                                  const int64_t *ts, int R, int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
+                                                  const SRC src, int R, int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
@@ -1594,13 +1682,14 @@ __global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBu
         if (status) status[b] = fst;
     }
     for (int p = tid; p < n; p += nt)
-        idx[(size_t)b * n + p] = fst == ZL_OK ? last_index_not_after(ts + ((size_t)b * n + p) * R, R, bar) : -1;
+        idx[(size_t)b * n + p] = fst == ZL_OK ? last_index_not_after(src.inst(b, n, R).row(p), R, bar) : -1;
 }
 
 // ------------------------------------------------------------------------------ finalize
 // grid (row blocks, B): every CTA reduces the instance's partial results, then recovers the indices of
 // its block of rows; the CTA of row block 0 also writes wait, barrier and status.
-__global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int R, int nseg, FilterBufs F, int nres,
+template <class SRC>
+__global__ void __launch_bounds__(256) k_finalize(const SRC src, int n, int R, int nseg, FilterBufs F, int nres,
                                                   int objective, int filter, const InstMeta *meta, const SegResult *seg,
                                                   int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
     grid_dep_wait();
@@ -1647,7 +1736,7 @@ __global__ void __launch_bounds__(256) k_finalize(const int64_t *ts, int n, int 
     if (p < n) {
         int res = -1;
         if (fst == ZL_OK) {
-            res = last_index_not_after(ts + ((size_t)b * n + p) * R, R, bar);
+            res = last_index_not_after(src.inst(b, n, R).row(p), R, bar);
         }
         idx[(size_t)b * n + p] = res;
     }
@@ -1940,10 +2029,14 @@ void launch_dep(bool early, void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
     cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_t *ev) {
+// SRC: zl::MatBatch (the rows are read from q.ts) or zl::AriBatch (predicted rows, generated on the fly; RANGE, filter
+// route or plain segment sweep only).
+template <class SRC>
+void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_t *ev, const SRC src) {
+    constexpr bool arith = std::is_same<SRC, zl::AriBatch>::value;
     const bool filter = q.fb.table != nullptr && q.objective == ZL_OBJ_RANGE;
     // the bucket route: every SUM shape it supports, and RANGE instances small enough to be a single bucket
-    const bool sumfast = q.fb.flags != nullptr && q.fb.scap != 0 && (q.objective == ZL_OBJ_SUM || q.fb.table == nullptr);
+    const bool sumfast = !arith && q.fb.flags != nullptr && q.fb.scap != 0 && (q.objective == ZL_OBJ_SUM || q.fb.table == nullptr);
     zl::FilterBufs fb = q.fb;
     if (!filter && !sumfast) memset(&fb, 0, sizeof(fb));
     if (ev) cudaEventRecord(ev[0], st);
@@ -1952,8 +2045,8 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     const int pthreads = q.prologue_threads ? q.prologue_threads
                          : many ? std::max(128, std::min(256, pow2_ceil(2 * q.n))) : std::max(512, std::min(1024, pow2_ceil(q.n)));
     // the first kernel of a call is scheduled early too: it waits (grid_dep_wait) for whatever precedes it in the stream
-    launch_dep(!((q.pdl_off >> 9) & 1), zl::k_prologue, dim3(q.B), dim3(pthreads), (size_t)q.n * 16, st, q.ts, q.n, q.R, q.objective, q.flags, q.meta, fb);
-    if (q.flags & ZL_FLAG_CHECK_SORTED) {
+    launch_dep(!((q.pdl_off >> 9) & 1), zl::k_prologue<SRC>, dim3(q.B), dim3(pthreads), (size_t)q.n * 16, st, src, q.n, q.R, q.objective, q.flags, q.meta, fb);
+    if (!arith && (q.flags & ZL_FLAG_CHECK_SORTED)) {
         const size_t total = (size_t)q.B * q.n * q.R;
         const int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)q.num_sms * 16);
         launch_dep(!((q.pdl_off >> 0) & 1), zl::k_check_sorted, dim3(blocks), dim3(256), 0, st, q.ts, q.n, q.R, total, q.meta);
@@ -1969,11 +2062,14 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         fb.nreg = (int)((q.n + rpc - 1) / rpc);
         fb.regcap = fb.list1cap / fb.nreg;
         const size_t fsmem = (size_t)fb.cells * 4 + (size_t)nw * zl::FILTER_STAGES * zl::FILTER_SLOT * 8;
-        launch_dep(!((q.pdl_off >> 1) & 1), zl::k_filter, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.flags, (int)rpc, q.filter_round ? q.filter_round : 8, q.meta, fb);
+        if constexpr (arith)
+            launch_dep(!((q.pdl_off >> 1) & 1), zl::k_filter_arith, dim3(fb.nreg, q.B), dim3(threads), (size_t)fb.cells * 4, st, src, q.n, q.R, (int)rpc, q.meta, fb);
+        else
+            launch_dep(!((q.pdl_off >> 1) & 1), zl::k_filter, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.flags, (int)rpc, q.filter_round ? q.filter_round : 8, q.meta, fb);
         if (ev) cudaEventRecord(ev[2], st);
         const int tcap = (int)std::min<long long>((long long)zl::TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
-        launch_dep(!((q.pdl_off >> 2) & 1), zl::k_tail, dim3(q.B), dim3(q.tail_threads ? q.tail_threads : many ? (tcap <= 1024 ? 128 : 256) : std::max(64, std::min(1024, tcap / 2))), (size_t)tcap * 20 + (size_t)fb.cells * 4, st,
-                   (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg, tcap, q.ts, q.R, q.idx, q.barrier, q.wait, q.status);
+        launch_dep(!((q.pdl_off >> 2) & 1), zl::k_tail<SRC>, dim3(q.B), dim3(q.tail_threads ? q.tail_threads : many ? (tcap <= 1024 ? 128 : 256) : std::max(64, std::min(1024, tcap / 2))), (size_t)tcap * 20 + (size_t)fb.cells * 4, st,
+                   (const zl::InstMeta *)q.meta, fb, q.n, q.nres, q.seg, tcap, src, q.R, q.idx, q.barrier, q.wait, q.status);
         // the route for instances with many survivors: fixed-size grids that return at once when no instance needs them
         const int tiles = (fb.fcells + zl::SCAN_TILE - 1) / zl::SCAN_TILE;
         const int wide = 4 * q.num_sms;
@@ -2020,22 +2116,26 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     // with a fast route on, the segment sweep is only the fallback: a small persistent grid
     const int items = p.nseg * q.B;
     const int sweep_ctas = fast ? std::min(items, 2 * q.num_sms) : items;
-    if (q.objective == ZL_OBJ_RANGE) launch_dep(!((q.pdl_off >> 7) & 1), zl::k_sweep<ZL_OBJ_RANGE>, dim3(sweep_ctas), dim3(p.threads), p.smem, st, sp);
-    else launch_dep(!((q.pdl_off >> 7) & 1), zl::k_sweep<ZL_OBJ_SUM>, dim3(sweep_ctas), dim3(p.threads), p.smem, st, sp);
+    if (q.objective == ZL_OBJ_RANGE) launch_dep(!((q.pdl_off >> 7) & 1), zl::k_sweep<ZL_OBJ_RANGE, SRC>, dim3(sweep_ctas), dim3(p.threads), p.smem, st, sp, src);
+    else launch_dep(!((q.pdl_off >> 7) & 1), zl::k_sweep<ZL_OBJ_SUM, SRC>, dim3(sweep_ctas), dim3(p.threads), p.smem, st, sp, src);
     if (ev) cudaEventRecord(ev[3], st);
     const int fthreads = std::max(32, std::min(256, pow2_ceil(q.n)));
-    launch_dep(!((q.pdl_off >> 8) & 1), zl::k_finalize, dim3((q.n + fthreads - 1) / fthreads, q.B), dim3(fthreads), 0, st, q.ts, q.n, q.R, p.nseg, fb, q.nres, q.objective,
+    launch_dep(!((q.pdl_off >> 8) & 1), zl::k_finalize<SRC>, dim3((q.n + fthreads - 1) / fthreads, q.B), dim3(fthreads), 0, st, src, q.n, q.R, p.nseg, fb, q.nres, q.objective,
                                                                   filter ? 1 : sumfast ? 2 : 0, q.meta, q.seg, q.idx, q.barrier, q.wait, q.status);
     if (ev) cudaEventRecord(ev[4], st);
 }
 
 cudaError_t raise_shared_memory_limits() {
-    cudaError_t e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_RANGE, zl::MatBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_SUM, zl::MatBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_RANGE, zl::AriBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sweep<ZL_OBJ_SUM, zl::AriBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_buckets, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_tail, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_prologue, cudaFuncAttributeMaxDynamicSharedMemorySize, zl::MAX_WORKERS * 16);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_tail<zl::MatBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_tail<zl::AriBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_prologue<zl::MatBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, zl::MAX_WORKERS * 16);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_prologue<zl::AriBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, zl::MAX_WORKERS * 16);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_buckets<ZL_OBJ_SUM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_buckets<ZL_OBJ_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(zl::k_sum_plan, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
@@ -2326,7 +2426,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
     if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
-    enqueue(q, p, st, ev);
+    enqueue(q, p, st, ev, zl::MatBatch{d_ts});
     if (ev) ++h->prof_calls;
     ZL_CUDA(h, cudaGetLastError());
     h->launches += zl_launches_per_call(h);
@@ -2374,6 +2474,30 @@ zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const i
                                     void *cuda_stream) {
     if (!h || !h->d_pred) return ZL_ERR_INVALID_ARG;
     if (B < 1 || B > h->cfg.max_batch) return ZL_ERR_INVALID_ARG;
+    if (h->cfg.objective == ZL_OBJ_RANGE && h->fb.table != nullptr) {
+        // the filter route (and its fallback) on generated rows: the predicted matrix is never written
+        if (!d_last || !d_interval || !d_idx || !d_barrier || !d_wait) return ZL_ERR_INVALID_ARG;
+        if (((uintptr_t)d_last & 7) || ((uintptr_t)d_interval & 7) || ((uintptr_t)d_barrier & 7) || ((uintptr_t)d_wait & 7) ||
+            ((uintptr_t)d_idx & 3) || ((uintptr_t)d_status & 3))
+            return ZL_ERR_INVALID_ARG;
+        const LaunchPlan p = make_plan(h, B);
+        if (p.smem > 200 * 1024) return ZL_ERR_UNSUPPORTED;
+        cudaEvent_t *ev = (h->prof_ev && h->prof_calls < h->prof_cap) ? h->prof_ev + PROF_EVENTS * (size_t)h->prof_calls : nullptr;
+        Pipeline q;
+        q.ts = nullptr; q.B = B; q.n = h->cfg.n_workers; q.R = h->cfg.lookahead_R; q.objective = ZL_OBJ_RANGE;
+        q.flags = h->cfg.flags & ~ZL_FLAG_CHECK_SORTED; q.num_sms = h->num_sms;
+        q.meta = h->d_meta; q.seg = h->d_seg; q.nres = h->nres;
+        q.fb = h->fb;
+        q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.filter_round = h->opt_filter_round; q.pdl_off = h->opt_pdl_off;
+        q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
+        if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
+        q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
+        enqueue(q, p, (cudaStream_t)cuda_stream, ev, zl::AriBatch{d_last, d_interval});
+        if (ev) ++h->prof_calls;
+        ZL_CUDA(h, cudaGetLastError());
+        h->launches += zl_launches_per_call(h);
+        return ZL_OK;
+    }
     zl_status rc = zl_predict_batched(d_last, d_interval, B, h->cfg.n_workers, h->cfg.lookahead_R, h->d_pred, cuda_stream);
     if (rc != ZL_OK) return rc;
     ++h->launches;
@@ -2511,7 +2635,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     memset(&q.fb, 0, sizeof(q.fb));
     q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
-    enqueue(q, p, (cudaStream_t)cuda_stream, nullptr);
+    enqueue(q, p, (cudaStream_t)cuda_stream, nullptr, zl::MatBatch{d_ts});
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;
 }
 
