@@ -111,9 +111,13 @@ zl_status zl_predict_batched(const int64_t *d_last, const int64_t *d_interval, i
                              int64_t *d_ts, void *cuda_stream);
 
 /*
- * Both phases of ZipLine in one call: predict into the handle's own buffer (the handle must have been
- * created with ZL_FLAG_PREDICTOR, else ZL_ERR_INVALID_ARG), then the search of zl_select_batched on it.
- * Outputs, stream and error behaviour as for zl_select_batched.
+ * Both phases of ZipLine in one call (the handle must have been created with ZL_FLAG_PREDICTOR, else
+ * ZL_ERR_INVALID_ARG).  For the RANGE objective on shapes of more than 4096 timestamps the predicted matrix
+ * is never written: the kernels generate e^p_i = last[p] + i * interval[p] where they would read a row, and
+ * the filter pass settles a whole worker at once from its interval.  Otherwise (SUM, small shapes) the
+ * prediction goes into the handle's own buffer and zl_select_batched runs on it.  Same results either way;
+ * outputs, stream and error behaviour as for zl_select_batched (a worker with a negative input, or whose
+ * last prediction would reach 2^62, makes its instance ZL_ERR_INVALID_ARG).
  */
 zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const int64_t *d_interval, int32_t B,
                                     int32_t *d_idx, int64_t *d_barrier, int64_t *d_wait, int32_t *d_status,

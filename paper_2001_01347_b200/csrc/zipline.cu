@@ -34,6 +34,10 @@
 //               segments are independent.
 //
 //   k_finalize  minimum over an instance's partial results, barrier, per-worker index recovery.
+//
+// Predicted rows (e_i = last + (i + 1) * interval) need not exist in memory: k_prologue, k_sweep, k_tail and
+// k_finalize are templates over a row source (MatBatch reads the matrix, AriBatch computes the rule), and
+// k_filter_arith is the filter pass on such rows.
 //   k_trace     per-position intermediates of the steps for small instances (tests).
 #include <cuda_runtime.h>
 #include <stddef.h>
