@@ -2233,9 +2233,12 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         f.cells = std::max(64, std::min(zl::FILTER_MAX_CELLS, pow2_ceil((int)std::min<long long>(cfg->lookahead_R, 1 << 20))));
         f.capb = (int)std::max<long long>(64, std::min<long long>(4096, pow2_ceil((int)std::min<long long>(N, 1 << 20))));
         f.nbk = (int)std::max<long long>(1, std::min<long long>(1024, pow2_ceil((int)std::min<long long>(N / 8 / f.capb, 1 << 20))));
+        // small shapes: room for half of the instance's elements (at most four buckets), so that instances in which
+        // many elements raise the running maximum stay on this route
+        f.nbk = std::max(f.nbk, (int)std::min<long long>(4, pow2_ceil((int)std::max<long long>(1, N / 2 / f.capb))));
         f.fcells = (int)std::max<long long>(std::max(64, f.nbk), std::min<long long>(1 << 18, pow2_ceil((int)std::min<long long>(N / 64, 1 << 20))));
         f.grp = std::max(1, std::min(f.nbk, pow2_floor((int)std::max<long long>(1, (long long)f.nbk * cfg->max_batch / (8LL * std::max(1, h->num_sms))))));
-        f.list1cap = (int)std::max<long long>(N / 2, std::min<long long>(N, 4096));
+        f.list1cap = (int)(N <= (1 << 17) ? N : N / 2);            // small shapes: room for every element
         h->nres = std::max(zl::MAX_SEGMENTS, (f.nbk + f.grp - 1) / f.grp);
         const size_t tiles = ((size_t)f.fcells + zl::SCAN_TILE - 1) / zl::SCAN_TILE;
         const size_t sizes[9] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.fcells * 4, mb * cfg->n_workers * 4,
