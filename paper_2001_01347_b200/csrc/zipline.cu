@@ -141,6 +141,7 @@ struct FilterBufs {
     unsigned long long *cellacc;             // [B][scells + 1 + stiles*15 + 1]  scratch of the bucket plan
     uint16_t *itab;                          // [B][stiles][n][16]   per row: index of its first element in each bucket of the tile
     int32_t scells, sM, scap, stiles;        // scells == 0: every instance is a single bucket (n * R <= scap)
+    int32_t ssub;                            // set per call: CTAs that share the buckets of one tile (small batches)
 };
 
 struct SweepParams {
@@ -1372,8 +1373,11 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
     const bool single = F.scells == 0;
     const int per = max(1, nslots / nt);
     const int s0 = min(tid * per, nslots), s1 = min(s0 + per, nslots);
-    for (int item = blockIdx.x; item < F.stiles * B; item += gridDim.x) {
-        const int b = item / F.stiles, t = item - b * F.stiles;
+    // work item: (instance, tile, part of the tile); with few tiles in the batch a tile's buckets are shared out over
+    // ssub CTAs, each of which leaves a result of its own
+    const int per_inst = F.stiles * F.ssub;
+    for (int item = blockIdx.x; item < per_inst * B; item += gridDim.x) {
+        const int b = item / per_inst, ts_ = item - b * per_inst, t = ts_ / F.ssub, sub = ts_ - t * F.ssub;
         __syncthreads();                                          // shared state of the previous item is done with
         if (tid == 0) { sM = meta[b]; sstatus = 0; }              // one read: another CTA may set `overflow` meanwhile
         __syncthreads();
@@ -1383,10 +1387,12 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
         const uint32_t tminlo = (uint32_t)(uint64_t)M.tmin - 1u;
         const uint16_t *tab = single ? nullptr : F.itab + ((size_t)b * F.stiles + t) * n * 16;
         const uint32_t *bnd = single ? nullptr : F.bnd + (size_t)b * ((size_t)F.stiles * TILE_BK + 1) + (size_t)t * TILE_BK;
-        const int j1 = min(TILE_BK, (int)M.count - t * TILE_BK);  // buckets of this tile
+        const int jt = min(TILE_BK, (int)M.count - t * TILE_BK);  // buckets of this tile
+        const int jper = (TILE_BK + F.ssub - 1) / F.ssub;
+        const int j0 = sub * jper, j1 = min(jt, j0 + jper);         // ... and of this part of it (may be none)
         uint64_t bd = ~0ull, bt = ~0ull;
         bool over = false;
-        for (int j = 0; j < j1; ++j) {
+        for (int j = j0; j < j1; ++j) {
             for (int s = tid; s <= slot_pad(nslots); s += nt) cnt[s] = 0;
             if (tid == 0) { sh.fill = 0; sh.nlong = 0; sh.carryC = 0; sh.carryS = 0; }
             // times of the bucket lie in [lo, hi): slot = ((T - lo) * scale) >> 32 < nslots, monotone in T
@@ -1546,7 +1552,7 @@ __global__ void __launch_bounds__(1024) k_sum_buckets(const int64_t *ts, int n, 
             if (tid == 0) { meta[b].overflow = 1; F.flags[1] = 1; }
             continue;
         }
-        block_best_to_result(bd, bt, ZL_OK, tmpA, &sstatus, seg[(size_t)b * nres + t]);
+        block_best_to_result(bd, bt, ZL_OK, tmpA, &sstatus, seg[(size_t)b * nres + ts_]);
     }
 }
 
@@ -1711,7 +1717,7 @@ __global__ void __launch_bounds__(256) k_finalize(const SRC src, int n, int R, i
     uint32_t st = M.status;
     if (st == ZL_OK) {
         const int used = !handled_by_filter(M, filter) ? nseg
-                         : filter == 2 ? (int)M.count2                                  // bucket route: one result per tile
+                         : filter == 2 ? (int)M.count2 * F.ssub                         // bucket route: one result per part of a tile
                          : tail_instance(M) ? 1 : (F.nbk + bucket_group(F, M.count2) - 1) / bucket_group(F, M.count2);
         for (int s = tid; s < used; s += blockDim.x) {
             const SegResult r = seg[(size_t)b * nres + s];
@@ -2100,7 +2106,9 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         int bthreads = single ? (int)std::max<long long>(64, std::min<long long>(1024, pow2_ceil((int)((N + 7) / 8))))
                               : (fb.scap > 4096 ? 1024 : 512);
         if (q.tail_threads) bthreads = q.tail_threads;
-        const int items = fb.stiles * q.B;
+        // few tiles in the batch: share each tile's buckets out over several CTAs
+        fb.ssub = single ? 1 : std::max(1, std::min(zl::TILE_BK, (2 * q.num_sms) / std::max(1, fb.stiles * q.B)));
+        const int items = fb.stiles * fb.ssub * q.B;
         const size_t bsmem = (size_t)fb.scap * 18 + ((size_t)fb.scap + fb.scap / 32 + 2) * 4;
         if (q.objective == ZL_OBJ_SUM)
             launch_dep(!((q.pdl_off >> 3) & 1), zl::k_sum_buckets<ZL_OBJ_SUM>, dim3(std::min(items, 32 * q.num_sms)), dim3(bthreads), bsmem, st,
@@ -2273,7 +2281,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
                 if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
                 filter_b += sizes[i];
             }
-            h->nres = std::max(zl::MAX_SEGMENTS, f.stiles);
+            h->nres = std::max(zl::MAX_SEGMENTS, f.stiles * zl::TILE_BK);   // up to one result per bucket
         } else {
             memset(&f, 0, sizeof(f));
         }
