@@ -2085,7 +2085,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
         const int wide = 4 * q.num_sms;
         launch_dep(!((q.pdl_off >> 3) & 1), zl::k_tilemax, dim3(std::min(tiles * q.B, wide)), dim3(256), 0, st, (const zl::InstMeta *)q.meta, fb, q.B);
         launch_dep(!((q.pdl_off >> 4) & 1), zl::k_cellscan, dim3(std::min(tiles * q.B, wide)), dim3(256), 0, st, (const zl::InstMeta *)q.meta, fb, q.B);
-        launch_dep(!((q.pdl_off >> 5) & 1), zl::k_refine, dim3(std::min(fb.nreg * q.B, wide)), dim3(256), 0, st, q.meta, fb, q.B);
+        launch_dep(!((q.pdl_off >> 5) & 1), zl::k_refine, dim3(std::min(fb.nreg * q.B, 8 * wide)), dim3(256), 0, st, q.meta, fb, q.B);
         const int ngroups = (fb.nbk + fb.grp - 1) / fb.grp;
         const int bthreads = std::max(64, std::min(256, fb.capb / 4));
         launch_dep(!((q.pdl_off >> 6) & 1), zl::k_buckets, dim3(std::min(ngroups * q.B, wide)), dim3(bthreads), (size_t)fb.capb * 20, st,
