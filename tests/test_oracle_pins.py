@@ -147,6 +147,26 @@ def test_common_period_closed_form():
         assert o.sweep_window(M, o.RANGE)[0] == expect
 
 
+def test_common_period_closed_form_for_the_total_wait():
+    # same rows, SUM objective, R >= 3: while every row still has elements the total wait at time T is
+    # sum_p ((T - c_p) mod m), candidates are the element times, so the minimum is min_q sum_p ((c_q - c_p) mod m);
+    # after the rows run out the wait only grows.  The barrier is congruent to a minimising offset.
+    rng = np.random.default_rng(8)
+    for _ in range(200):
+        n = int(rng.integers(1, 9))
+        m = int(rng.integers(5, 400))
+        R = int(rng.integers(3, 9))
+        c = rng.integers(0, m, size=n)
+        M = c[:, None] + m * np.arange(R)[None, :]
+        totals = ((c[:, None] - c[None, :]) % m).sum(axis=1)           # totals[q] = sum_p ((c_q - c_p) mod m)
+        expect = int(totals.min())
+        for fn in (o.sweep, o.sweep_window):
+            wait, barrier, idx = fn(M, o.SUM)
+            assert wait == expect
+            assert barrier % m in set((c[totals == expect] % m).tolist())
+            assert barrier <= int(c.max()) + m                           # the first minimum comes within one period
+
+
 # ------------------------------------------------------------------ invariants of the definition
 def _rand_rows(rng, n, R, hi=500):
     return rng.integers(0, hi, size=(n, 1)) + np.cumsum(rng.integers(0, hi, size=(n, R)), axis=1)
