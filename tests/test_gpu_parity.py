@@ -381,6 +381,30 @@ def test_sum_mixed_batch_of_routes():
     assert_same(ts, 1, got)
 
 
+# ---------------------------------------------------------------- closed forms at a size no CPU check needs
+def test_common_period_closed_forms_at_scale():
+    # rows c_p + i * m with one period: RANGE = m - largest circular gap of the offsets, SUM = min_q sum_p ((c_q - c_p) mod m)
+    rng = np.random.default_rng(2024)
+    for n, R, m in ((1500, 600, 1_000_003), (4000, 64, 50_021), (300, 3000, 997)):
+        B = 2
+        c = rng.integers(0, m, size=(B, n))
+        ts = (c[:, :, None] + m * np.arange(R)[None, None, :]).astype(np.int64)
+        for objective in OBJ:
+            idx, barrier, wait, status = gpu_select(ts, objective)
+            assert (status == 0).all()
+            for b in range(B):
+                if objective == 0:
+                    u = np.unique(c[b])
+                    gaps = np.diff(np.concatenate([u, [u[0] + m]]))
+                    expect = 0 if len(u) == 1 else m - int(gaps.max())
+                else:
+                    expect = int(((c[b][:, None] - c[b][None, :]) % m).sum(axis=1).min())
+                assert int(wait[b]) == expect, (n, R, m, objective, b)
+                chosen = ts[b][np.arange(n), idx[b]]
+                assert chosen.max() == barrier[b]
+                assert wait[b] == (barrier[b] - chosen.min() if objective == 0 else (barrier[b] - chosen).sum())
+
+
 # ---------------------------------------------------------------- extreme shapes
 @pytest.mark.parametrize("objective", OBJ)
 def test_extreme_aspect_ratios(objective):
