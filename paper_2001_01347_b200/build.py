@@ -1,18 +1,27 @@
-"""Compile the CUDA library in-tree with nvcc for sm_100a."""
+"""Compile the CUDA library in-tree with nvcc for sm_100a (one object per source file, then one shared library)."""
 from __future__ import annotations
 
+import glob
 import os
 import shutil
 import subprocess
+from concurrent.futures import ThreadPoolExecutor
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
+OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(_HERE, "libzipline.so")
-SOURCES = [os.path.join(CSRC, "zipline.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, "zl_device.cuh"),
-                  os.path.join(os.path.dirname(_HERE), "include", "zipline.h")]
-NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-shared", "-Xcompiler", "-fPIC"]
+INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
+NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC"]
+
+
+def sources() -> list[str]:
+    return sorted(glob.glob(os.path.join(CSRC, "*.cu")))
+
+
+def headers() -> list[str]:
+    return sorted(glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h"))
+                  + glob.glob(os.path.join(INCLUDE, "*.h")))
 
 
 def _nvcc() -> str:
@@ -22,18 +31,40 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found: the ZipLine CUDA library cannot be built")
 
 
+def _obj(src: str) -> str:
+    return os.path.join(OBJ, os.path.basename(src)[:-3] + ".o")
+
+
 def is_stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    return any(os.path.getmtime(d) > t for d in DEPS)
+    return any(os.path.getmtime(d) > t for d in sources() + headers())
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
     """Build ``libzipline.so`` next to this file when missing or older than its sources."""
-    if force or is_stale():
-        tmp = LIB + f".tmp{os.getpid()}"
-        cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES
-        subprocess.run(cmd, check=True, cwd=CSRC)
-        os.replace(tmp, LIB)
+    if not (force or is_stale()):
+        return LIB
+    nvcc = _nvcc()
+    os.makedirs(OBJ, exist_ok=True)
+    newest_header = max(os.path.getmtime(h) for h in headers())
+    todo = [s for s in sources()
+            if force or not os.path.exists(_obj(s)) or os.path.getmtime(_obj(s)) < max(os.path.getmtime(s), newest_header)]
+
+    def compile_one(src: str):
+        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", "-o", _obj(src), src]
+        return subprocess.run(cmd, cwd=CSRC, capture_output=True, text=True)
+
+    with ThreadPoolExecutor(max(1, min(len(todo), 4, os.cpu_count() or 1))) as ex:
+        results = list(ex.map(compile_one, todo))
+    for src, r in zip(todo, results):
+        if verbose or r.returncode != 0:
+            print(f"--- {os.path.basename(src)}\n{r.stdout}{r.stderr}", flush=True)
+        if r.returncode != 0:
+            raise RuntimeError(f"nvcc failed on {src}")
+    tmp = LIB + f".tmp{os.getpid()}"
+    subprocess.run([nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp] + [_obj(s) for s in sources()],
+                   check=True, cwd=CSRC)
+    os.replace(tmp, LIB)
     return LIB

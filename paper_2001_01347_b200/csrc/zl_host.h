@@ -1,0 +1,77 @@
+// Host side shared by the translation units: what one call enqueues (Pipeline), the launch plan of the
+// segment sweep, the launch helper, and the stage launchers each kernel file exports.  Every kernel is
+// launched from the file that defines it.
+#pragma once
+#include <cuda_runtime.h>
+#include <string.h>
+
+#include <algorithm>
+
+#include "zl_types.cuh"
+
+namespace zl {
+
+inline int pow2_floor(int x) { int p = 1; while (p * 2 <= x) p *= 2; return p; }
+inline int pow2_ceil(int x) { int p = 1; while (p < x) p *= 2; return p; }
+
+// Shape of the segment sweep for one call.
+struct LaunchPlan { int threads, G, nseg, cap, target; size_t smem; };
+
+// Everything one call enqueues, for both the handle-based and the fixed-scratch entry points.
+struct Pipeline {
+    const int64_t *ts; int B, n, R, objective, flags, num_sms;
+    InstMeta *meta; SegResult *seg; int nres;
+    FilterBufs fb;                                                // fb.table == nullptr: no filter route
+    int filter_threads, filter_rows, filter_round;                // 0: automatic
+    int pdl_off;                                                  // bit mask of kernels launched without early scheduling
+    int prologue_threads, tail_threads;                           // 0: automatic
+    int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;
+};
+
+// Launch with programmatic stream serialization: the kernel may be scheduled while its predecessor in
+// the stream is still running; every kernel here waits for that predecessor (grid_dep_wait) before it
+// touches memory.
+template <typename... KArgs, typename... Args>
+void launch_dep(bool early, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = early ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// ---- stage launchers.  `fb` is the call's copy of the route buffers (all zero when no fast route is on);
+// the filter and bucket stages fill in its per-call fields.  Each *_limits() raises the dynamic shared-memory
+// limit of its file's kernels (once per device).
+
+// prologue.cu: column scans (+ filter table), optional sortedness check
+void enqueue_prologue(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const MatBatch &src);
+void enqueue_prologue(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const AriBatch &src);
+cudaError_t prologue_limits();
+
+// filter.cu: RANGE filter pass and the single-CTA finish of instances with few survivors; `mid` (may be null)
+// is recorded between the two
+void enqueue_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid, const MatBatch &src);
+void enqueue_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid, const AriBatch &src);
+cudaError_t filter_limits();
+
+// heavy.cu: RANGE instances with many survivors (cell scan, refinement, bucket sweep)
+void enqueue_heavy(const Pipeline &q, const FilterBufs &fb, cudaStream_t st);
+cudaError_t heavy_limits();
+
+// sum_route.cu: the bucket route (plan, index pass, bucket kernel); `mid` is recorded before the bucket kernel
+void enqueue_bucket_route(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid);
+cudaError_t bucket_route_limits();
+
+// sweep.cu: the segment sweep (fallback of the fast routes, or the whole search) and K5
+void enqueue_sweep(const Pipeline &q, const FilterBufs &fb, const LaunchPlan &p, bool fast, cudaStream_t st, const MatBatch &src);
+void enqueue_sweep(const Pipeline &q, const FilterBufs &fb, const LaunchPlan &p, bool fast, cudaStream_t st, const AriBatch &src);
+// route: 0 only the segment sweep ran, 1 the RANGE filter route, 2 the bucket route
+void enqueue_finalize(const Pipeline &q, const FilterBufs &fb, const LaunchPlan &p, int route, cudaStream_t st, const MatBatch &src);
+void enqueue_finalize(const Pipeline &q, const FilterBufs &fb, const LaunchPlan &p, int route, cudaStream_t st, const AriBatch &src);
+cudaError_t sweep_limits();
+
+}  // namespace zl
