@@ -4,9 +4,12 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
                     [--workload c4] [--objective range|sum]
 
-A step is one pass of the whole hot path (prologue, sweep, finalize) over one batch of synthetic
-input.  The default workload is the n=1024, R=1024, B=64 configuration (512 MiB of int64
-timestamps per step, larger than L2).  One JSON line is printed by rank 0.
+A step is one pass of the whole hot path (one ``zl_select_batched`` call) over one batch of synthetic
+input.  The default workload is the n=1024, R=1024, B=64 configuration (512 MiB of int64 timestamps per
+step).  Each of the K timed steps is measured with its own pair of CUDA events around ``inner`` consecutive
+calls (so that the timed region lasts at least 0.1 s whatever K is) and reported as time per call; the
+inputs rotate over as many copies as it takes for the bytes a call examines, times the copies, to exceed
+the L2 several times over.  One JSON line is printed by rank 0.
 
 With N > 1 (launched through torch.distributed.run) every rank runs the same-sized batch on its
 own GPU with its own instance seeds: the batch dimension shards, there is no data-path
@@ -15,6 +18,7 @@ collective, and ``value`` is the sum over ranks divided by the slowest rank's ti
 from __future__ import annotations
 
 import argparse
+import glob
 import json
 import os
 import statistics
@@ -30,7 +34,9 @@ if ROOT not in sys.path:
 
 import zl_inputs  # noqa: E402
 
-METRIC = "ZipLine timestamps/sec (selections/sec in config) at 1 B200; achieved HBM GB/s vs peak"
+METRIC = "ZipLine timestamps/sec (selections/sec in result) at 1 B200; achieved HBM GB/s vs peak"
+NOMINAL_GBS = 8000.0                   # the HBM3e figure the target is quoted against
+MIN_TIMED_MS = 100.0
 CLOCK_QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -41,14 +47,15 @@ def recorded_traffic(key):
     import hashlib
     try:
         rec = {}
-        with open(os.path.join(ROOT, "profiles", "k_filter_c4_traffic.txt")) as f:
+        with open(os.path.join(ROOT, "profiles", "traffic.txt")) as f:
             for line in f:
                 if line.strip() and not line.startswith("#"):
                     k, v = line.split()
                     rec[k] = v
         hsh = hashlib.sha256()
-        for name in ("zipline.cu", "zl_device.cuh"):
-            with open(os.path.join(ROOT, "paper_2001_01347_b200", "csrc", name), "rb") as f:
+        csrc = os.path.join(ROOT, "paper_2001_01347_b200", "csrc")
+        for path in sorted(glob.glob(os.path.join(csrc, "*.cu")) + glob.glob(os.path.join(csrc, "*.cuh")) + glob.glob(os.path.join(csrc, "*.h"))):
+            with open(path, "rb") as f:
                 hsh.update(f.read())
         return int(rec[key]) if rec.get("source_sha256") == hsh.hexdigest() and key in rec else None
     except Exception:
@@ -112,67 +119,81 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def oracle_sample(ts: np.ndarray, objective: int, max_instances: int, budget_s: float):
-    """Time the oracle's sweep on up to max_instances instances, one thread per host core."""
+def oracle_sample(ts: np.ndarray, objective: int, instances: int):
+    """Time the oracle's sweep on the first `instances` instances, one thread per host core."""
     from concurrent.futures import ThreadPoolExecutor
 
     import oracle
     cores = os.cpu_count() or 1
-    B = min(ts.shape[0], max_instances)
-    t_one = time.perf_counter()
-    oracle.sweep_window(ts[0], objective)                       # also sizes the sample
-    t_one = time.perf_counter() - t_one
-    B = max(1, min(B, int(budget_s * cores / max(t_one, 1e-6))))
-    threads = min(cores, B)
+    threads = min(cores, instances)
     t0 = time.perf_counter()
     with ThreadPoolExecutor(threads) as ex:
-        list(ex.map(lambda b: oracle.sweep_window(ts[b], objective), range(B)))
-    dt = time.perf_counter() - t0
-    return B, threads, dt
+        list(ex.map(lambda b: oracle.sweep_window(ts[b], objective), range(instances)))
+    return threads, time.perf_counter() - t0
 
 
-def run_reference(args, w, objective):
-    """The oracle, as it stands, on the host cores (rank 0 only)."""
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
-    ts = zl_inputs.generate(w, B=min(w.B, 16))
-    per_step = []
-    used = (0, 0)
-    for s in range(args.warmup + args.steps):
-        B, threads, dt = oracle_sample(ts, objective, max_instances=16, budget_s=4.0)
-        used = (B, threads)
-        if s >= args.warmup:
-            per_step.append(dt / B)                             # seconds per instance
-    sec_inst = statistics.mean(per_step)
-    value = w.n * w.R / sec_inst
-    sample = f"{used[0]} of {w.B} instances of {w.name} per step, sweep_window, {used[1]} threads"
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "timestamps/s", "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_inst * w.B * 1e3,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
-            "data": "synthetic", "config": workload_config(w, objective, args.gpus),
-            "cpu_baseline": {"value": value, "unit": "timestamps/s", "cores": used[1], "kind": "oracle", "sample": sample},
-            "e2e": {"value": value, "unit": "timestamps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
-    print(json.dumps(line), flush=True)
+def oracle_sample_size(ts: np.ndarray, objective: int, budget_s: float) -> int:
+    """How many instances of the batch the oracle gets through in about budget_s seconds on the host cores."""
+    import oracle
+    t = time.perf_counter()
+    oracle.sweep_window(ts[0], objective)
+    t = max(time.perf_counter() - t, 1e-6)
+    return max(1, min(ts.shape[0], int(budget_s * (os.cpu_count() or 1) / t)))
 
 
 def workload_config(w, objective, gpus):
     return {"workload": f"{w.name}: n={w.n} workers, R={w.R} lookahead, B={w.B} instances per GPU per step",
             "n": w.n, "R": w.R, "B": w.B, "objective": "range" if objective == 0 else "sum",
-            "input_bytes_per_step_per_gpu": w.timestamps * 8, "l2": "inputs larger than L2 (no flush needed)"
-            if w.timestamps * 8 > 200e6 else "inputs rotate over copies larger than L2",
+            "input_bytes_per_step_per_gpu": w.timestamps * 8,
+            "l2": "inputs rotate over copies so that the bytes one call examines x copies exceed 300 MB (more than twice the L2)",
             "parallelism": f"batch sharded over {gpus} GPU(s), no collective"}
+
+
+def run_reference(args, w, objective):
+    """The oracle, as it stands, on the host cores (rank 0 only): every step sweeps the same bounded sample of the batch."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    ts = zl_inputs.generate(w)
+    total = max(1, args.steps + args.warmup)
+    inst = oracle_sample_size(ts, objective, budget_s=min(8.0, 120.0 / total))
+    per_step, threads = [], 1
+    for s in range(args.warmup + args.steps):
+        threads, dt = oracle_sample(ts, objective, inst)
+        if s >= args.warmup:
+            per_step.append(dt)
+    sec = statistics.median(per_step)
+    value = inst * w.n * w.R / sec
+    sample = f"the first {inst} of {w.B} instances of {w.name} per step, sweep_window (sort + one pass), {threads} threads"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "timestamps/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
+            "data": "synthetic", "config": workload_config(w, objective, args.gpus),
+            "timing": {"ms_per_step_median": sec * 1e3, "ms_per_step_min": min(per_step) * 1e3, "ms_per_step_max": max(per_step) * 1e3,
+                       "what": "one step = the oracle on the sample named in cpu_baseline.sample (not extrapolated to the batch)"},
+            "cpu_baseline": {"value": value, "unit": "timestamps/s", "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "timestamps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+STAGES = {  # names of what runs between the library's stage events, by (route, cluster kernel)
+    (1, True): ("-", "k_range_fused", "k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep", "k_finalize"),
+    (1, False): ("k_prologue", "k_filter", "k_tail+k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep", "k_finalize"),
+    (2, False): ("k_prologue", "k_sum_plan+k_sum_index", "k_sum_buckets+k_sweep", "k_finalize"),
+    (0, False): ("k_prologue", "-", "k_sweep", "k_finalize"),
+}
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="zipline", choices=["zipline", "reference"])
     ap.add_argument("--workload", default="c4")
     ap.add_argument("--objective", default="range", choices=["range", "sum"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-probe", action="store_true")
     ap.add_argument("--opt", action="append", default=[], help="library option key=value")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "zipline" else args.warmup
@@ -200,12 +221,9 @@ def main():
 
     # ---- inputs: this rank's shard of the global batch (instances rank*B .. rank*B+B-1)
     ts_np = zl_inputs.generate(w, first_instance=rank * w.B)
-    copies = max(1, int(np.ceil(300e6 / ts_np.nbytes)))        # rotate when one batch would fit in L2
-    d_ts = [torch.from_numpy(ts_np).to(dev)]
-    for c in range(1, copies):
-        d_ts.append(d_ts[0].clone())
-    h_pinned = torch.from_numpy(ts_np).pin_memory()
     nts = w.timestamps
+    lmin_inst = ts_np[:, :, -1].min(axis=1)
+    examined_early = int((ts_np <= lmin_inst[:, None, None]).sum())      # timestamps not after the first exhausted row
 
     def make_handle(flags):
         h = zl.ZipLine(w.n, w.R, w.B, objective, local, flags)
@@ -214,97 +232,124 @@ def main():
             h.set_option(k, int(v))
         return h
 
-    def timed(h, steps, warmup, host=False, profile=False):
+    h = make_handle(0)
+    route = h.route                                  # 0 segment sweep only, 1 RANGE filter route, 2 bucket route
+    cluster = bool(h.uses_cluster_kernel)
+    examined = examined_early if route == 1 else nts
+    copies = max(1, min(16, int(np.ceil(300e6 / (examined * 8)))))
+    d_ts = [torch.from_numpy(ts_np).to(dev)]
+    for c in range(1, copies):
+        d_ts.append(d_ts[0].clone())
+    h_pinned = torch.from_numpy(ts_np).pin_memory()
+
+    def timed(h, steps, warmup, host=False, profile=False, inner=None):
+        """Per-step times (ms per call) of `steps` samples of `inner` calls each; inner is sized from the warm-up."""
         sel = None
+        k = 0
 
-        def step(i):
-            nonlocal sel
-            sel = h.select_batched_host(h_pinned, sel) if host else h.select_batched(d_ts[i % copies], sel)
+        def call():
+            nonlocal sel, k
+            sel = h.select_batched_host(h_pinned, sel) if host else h.select_batched(d_ts[k % copies], sel)
+            k += 1
 
-        for i in range(warmup):
-            step(i)
+        for _ in range(warmup):
+            call()
         torch.cuda.synchronize()
+        if inner is None:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(8):
+                call()
+            b.record()
+            torch.cuda.synchronize()
+            est_ms = a.elapsed_time(b) / 8
+            inner = 1 if host else max(1, int(np.ceil(1.3 * MIN_TIMED_MS / (steps * est_ms))))
         if world > 1:
             dist.barrier()
             torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if profile:
-            h.profile_begin(steps)
+            h.profile_begin(steps * inner)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
         t0 = time.perf_counter()
-        e0.record()
-        for i in range(steps):
-            step(i)
-        e1.record()
+        for a, b in ev:
+            a.record()
+            for _ in range(inner):
+                call()
+            b.record()
         torch.cuda.synchronize()
         wall_ms = (time.perf_counter() - t0) * 1e3
-        ms = wall_ms if host else e0.elapsed_time(e1)          # the host path runs on the library's own stream
+        if host:                                                  # the host path runs on the library's own stream
+            per = [wall_ms / steps] * steps
+            total = wall_ms
+        else:
+            per = [a.elapsed_time(b) / inner for a, b in ev]
+            total = ev[0][0].elapsed_time(ev[-1][1])
         prof = None
         if profile:
             prof = h.profile_read()
             h.profile_end()
         if world > 1:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            t = torch.tensor([total], device=dev, dtype=torch.float64)
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+            total = float(t.item())
             dist.barrier()
-        return ms, prof, sel
+        return {"per": per, "total_ms": total, "inner": inner, "calls": steps * inner, "prof": prof, "sel": sel}
+
+    def spread(t):
+        return {"inner_repeats": t["inner"], "samples": len(t["per"]), "timed_region_ms": t["total_ms"],
+                "ms_per_step_median": statistics.median(t["per"]), "ms_per_step_min": min(t["per"]), "ms_per_step_max": max(t["per"])}
 
     sampler = ClockSampler(local)
-    h = make_handle(0)
     sampler.start()
-    ms, _, sel = timed(h, args.steps, args.warmup)                       # the headline: no per-stage events in the stream
-    psteps = max(3, min(args.steps, 50))
-    _, prof, _ = timed(h, psteps, 3, profile=True)                       # per-stage CUDA events (they serialise the stages)
-    status_ok = bool((sel.status == 0).all().item())
-    launches = h.launches_per_call * args.steps
-    ms_step = ms / args.steps
+    t_main = timed(h, args.steps, args.warmup)                           # the headline: no per-stage events in the stream
+    t_prof = timed(h, max(3, min(args.steps, 20)), 3, profile=True, inner=max(1, t_main["inner"] // 4))   # stage events serialise the stages
+    status_ok = bool((t_main["sel"].status == 0).all().item())
+    launches = h.launches_per_call * t_main["calls"]
+    ms_step = t_main["total_ms"] / t_main["calls"]
     value = world * nts / (ms_step * 1e-3)
 
     # the same search when every timestamp is examined (no early stop)
     hf = make_handle(zl.ZL_FLAG_FULL_SWEEP)
-    steps_f = max(3, args.steps // 2)
-    ms_f, _, _ = timed(hf, steps_f, 3)
-    _, prof_f, _ = timed(hf, psteps, 3, profile=True)
+    t_full = timed(hf, max(3, args.steps // 2), 3)
+    t_fprof = timed(hf, max(3, min(args.steps, 20)), 3, profile=True, inner=max(1, t_full["inner"] // 4))
     hf.destroy()
     clocks = sampler.stop()
+    ms_full = t_full["total_ms"] / t_full["calls"]
 
     # what the memory system delivers for the bytes of the filter pass: a kernel that only loads them (a warp per row, the
-    # row prefixes the early stop needs, then whole rows), with the L2 flushed before each launch and as run back to back
+    # row prefixes the early stop needs, then whole rows), over the same rotating copies
     probe = None
-    if rank == 0 and h.route == 1:
-        lmin_row = ts_np[:, :, -1].min(axis=1)
-        cnt = (ts_np <= lmin_row[:, None, None]).sum(axis=2).astype(np.int64)
+    if rank == 0 and route == 1 and not args.no_probe:
+        cnt = (ts_np <= lmin_inst[:, None, None]).sum(axis=2).astype(np.int64)
         pref = np.minimum(w.R, (cnt + 8 + 7) // 8 * 8).astype(np.int32).reshape(-1)     # as the filter pass requests them
         d_pref = torch.from_numpy(pref).to(dev)
         d_full = torch.full_like(d_pref, w.R)
         sink = torch.zeros(1, dtype=torch.int64, device=dev)
-        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
 
-        def probe_us(counts, cold, reps=10):
-            tot = 0.0
+        def probe_us(counts, reps=10, inner=8):
+            best = []
+            k = 0
             for i in range(reps + 2):
-                if cold:
-                    flush.zero_()
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 a.record()
-                zl.zl_probe_read_batched(d_ts[i % copies], counts, sink)
+                for _ in range(inner):
+                    zl.zl_probe_read_batched(d_ts[k % copies], counts, sink)
+                    k += 1
                 b.record()
                 torch.cuda.synchronize()
                 if i >= 2:
-                    tot += a.elapsed_time(b)
-            return tot / reps * 1e3
-        probe = {"prefix_bytes": int(pref.astype(np.int64).sum()) * 8,
-                 "prefix_us_cold_l2": probe_us(d_pref, True), "prefix_us": probe_us(d_pref, False),
-                 "full_bytes": nts * 8, "full_us_cold_l2": probe_us(d_full, True), "full_us": probe_us(d_full, False),
+                    best.append(a.elapsed_time(b) / inner * 1e3)
+            return statistics.median(best)
+        probe = {"prefix_bytes": int(pref.astype(np.int64).sum()) * 8, "prefix_us": probe_us(d_pref),
+                 "full_bytes": nts * 8, "full_us": probe_us(d_full),
                  "what": "load-only kernel on the bytes of the filter pass (row prefixes up to the first exhausted row, "
-                         "then whole rows); cold = 256 MB written before each launch"}
-        del flush
+                         "then whole rows), a warp per row, back to back over the rotating input copies"}
 
     # end to end: host buffers in, host results out, through the C ABI
     e2e_steps = max(3, min(args.steps, 10))
-    ms_e, _, _ = timed(h, e2e_steps, 3, host=True)
-    e2e_value = world * nts / (ms_e / e2e_steps * 1e-3)
-    h_route = h.route
+    t_e2e = timed(h, e2e_steps, 3, host=True)
+    ms_e2e = t_e2e["total_ms"] / t_e2e["calls"]
+    e2e_value = world * nts / (ms_e2e * 1e-3)
     h.destroy()
 
     if rank != 0:
@@ -312,56 +357,58 @@ def main():
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel (the sweep), algorithmic bytes = 8 per timestamp it must examine
+    # ---- roofline of the dominant kernel: algorithmic bytes = 8 per timestamp it must examine
     peak, peak_kind = measured_peak_gbs()
-    lmin = ts_np[:, :, -1].min(axis=1)
-    route = h_route                                  # 0 segment sweep only, 1 RANGE filter route, 2 bucket route
-    examined = int((ts_np <= lmin[:, None, None]).sum()) if route == 1 else nts
-    def dominant(pr):
-        if route == 1:
-            names = ("k_prologue", "k_filter", "k_tail+k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep", "k_finalize")
-        elif route == 2:
-            names = ("k_prologue", "k_sum_plan+k_sum_index", "k_sum_buckets+k_sweep", "k_finalize")
-        else:
-            names = ("k_prologue", "-", "k_sweep", "k_finalize")
-        stages = dict(zip(names, (pr["ms_prologue"], pr["ms_filter"], pr["ms_sweep"], pr["ms_finalize"])))
-        name = max(stages, key=stages.get)
-        return name, stages[name] / pr["calls"]
+    names = STAGES[(route, cluster)]
 
-    dom, sweep_ms = dominant(prof)
-    ach = examined * 8 / (sweep_ms * 1e-3) / 1e9
-    dom_f, sweep_ms_f = dominant(prof_f)
-    ach_f = nts * 8 / (sweep_ms_f * 1e-3) / 1e9
+    def dominant(pr):
+        stages = dict(zip(names, (pr["ms_prologue"], pr["ms_filter"], pr["ms_sweep"], pr["ms_finalize"])))
+        stages.pop("-", None)
+        name = max(stages, key=stages.get)
+        return name, stages[name] / pr["calls"], {k: v / pr["calls"] for k, v in stages.items()}
+
+    def fractions(nbytes, ms):
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        return {"GB/s": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8000": gbs / NOMINAL_GBS}
+
+    dom, dom_ms, stage_ms = dominant(t_prof["prof"])
+    ach = examined * 8 / (dom_ms * 1e-3) / 1e9
+    dom_f, dom_ms_f, stage_ms_f = dominant(t_fprof["prof"])
+    ach_f = nts * 8 / (dom_ms_f * 1e-3) / 1e9
+    model = ("8 B per timestamp not after the first exhausted row (the search stops there)" if route == 1 else "8 B per timestamp")
     roofline = {"bound": "hbm", "kernel": dom, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
-                "peak_kind": f"{peak_kind} copy bandwidth",
+                "peak_kind": f"{peak_kind} copy bandwidth", "frac_of_nominal_8000": ach / NOMINAL_GBS,
                 "traffic": recorded_traffic(f"{w.name}_{args.objective}_default_{dom}"),
-                "bytes_per_launch": examined * 8, "ms_per_launch": sweep_ms,
-                "bytes_model": "8 B per timestamp not after the first exhausted row (the search stops there)"
-                if route == 1 else "8 B per timestamp"}
-    full = {"value": nts / (ms_f / steps_f * 1e-3), "unit": "timestamps/s", "ms_per_step": ms_f / steps_f,
+                "bytes_per_launch": examined * 8, "ms_per_launch": dom_ms, "bytes_model": model,
+                "whole_call": {"examined_bytes": fractions(examined * 8, ms_step), "all_input_bytes": fractions(nts * 8, ms_step),
+                               "what": "the same bytes divided by ms_per_step (every kernel of the call, launch gaps included)"}}
+    full = {"value": world * nts / (ms_full * 1e-3), "unit": "timestamps/s", "ms_per_step": ms_full, "timing": spread(t_full),
+            "what": "ZL_FLAG_FULL_SWEEP: every timestamp is examined, so timestamps/s and bytes/s count the same elements",
             "roofline": {"bound": "hbm", "kernel": dom_f, "achieved": ach_f, "peak": peak, "unit": "GB/s",
-                         "frac": ach_f / peak, "bytes_per_launch": nts * 8, "ms_per_launch": sweep_ms_f,
-                         "traffic": recorded_traffic(f"{w.name}_{args.objective}_full_{dom_f}")}}
+                         "frac": ach_f / peak, "frac_of_nominal_8000": ach_f / NOMINAL_GBS, "bytes_per_launch": nts * 8,
+                         "ms_per_launch": dom_ms_f, "traffic": recorded_traffic(f"{w.name}_{args.objective}_full_{dom_f}"),
+                         "whole_call": {"all_input_bytes": fractions(nts * 8, ms_full)}},
+            "kernel_ms": stage_ms_f}
 
     cpu = None
     if not args.no_cpu_baseline and world == 1:
-        Bs, threads, dt = oracle_sample(ts_np, objective, max_instances=w.B, budget_s=20.0)
-        cpu = {"value": Bs * w.n * w.R / dt, "unit": "timestamps/s", "cores": threads, "kind": "oracle",
-               "sample": f"{Bs} of {w.B} instances of {w.name}, sweep_window (sort + one pass), {dt:.1f} s wall"}
+        inst = oracle_sample_size(ts_np, objective, budget_s=20.0)
+        threads, dt = oracle_sample(ts_np, objective, inst)
+        cpu = {"value": inst * w.n * w.R / dt, "unit": "timestamps/s", "cores": threads, "kind": "oracle",
+               "sample": f"the first {inst} of {w.B} instances of {w.name}, sweep_window (sort + one pass), {dt:.1f} s wall"}
 
-    cfg = workload_config(w, objective, world)
-    cfg.update({"selections_per_s": world * w.B / (ms_step * 1e-3), "early_stop": route == 1,
-                "route": {0: "segment sweep", 1: "filter", 2: "buckets"}[route],
-                "examined_fraction": examined / nts, "segments_per_instance": None,
-                "kernel_ms": {k[3:]: prof[k] / prof["calls"] for k in ("ms_prologue", "ms_filter", "ms_sweep", "ms_finalize")},
-                "kernel_ms_full_sweep": {k[3:]: prof_f[k] / prof_f["calls"]
-                                         for k in ("ms_prologue", "ms_filter", "ms_sweep", "ms_finalize")},
-                "all_status_ok": status_ok, "options": args.opt})
+    result = {"selections_per_s": world * w.B / (ms_step * 1e-3), "early_stop": route == 1,
+              "route": {0: "segment sweep", 1: "filter", 2: "buckets"}[route], "cluster_kernel": cluster,
+              "examined_fraction": examined / nts, "input_copies": copies,
+              "value_counts": "all n*R*B timestamps of the batch per call (nominal: the early stop examines examined_fraction of them; "
+                              "full_sweep.value counts examined timestamps only)",
+              "kernel_ms": stage_ms, "all_status_ok": status_ok, "options": args.opt}
     line = {"metric": METRIC, "value": value, "unit": "timestamps/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "int64", "data": "synthetic", "config": cfg, "clocks": clocks,
+            "vs_baseline": None, "dtype": "int64", "data": "synthetic", "config": workload_config(w, objective, world),
+            "timing": spread(t_main), "result": result, "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": "timestamps/s", "h2d_bytes_per_step": nts * 8,
-                    "d2h_bytes_per_step": w.B * (4 * w.n + 20), "ms_per_step": ms_e / e2e_steps},
+                    "d2h_bytes_per_step": w.B * (4 * w.n + 20), "ms_per_step": ms_e2e},
             "gpu_launches": launches, "roofline": roofline, "full_sweep": full, "cpu_baseline": cpu,
             "load_only_probe": probe}
     print(json.dumps(line), flush=True)

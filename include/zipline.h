@@ -43,7 +43,9 @@ typedef enum {
 enum {
     ZL_FLAG_CHECK_SORTED = 1,  /* verify every row is non-decreasing (one extra pass over the input) */
     ZL_FLAG_FULL_SWEEP = 2,    /* examine every timestamp even where the search could stop early    */
-    ZL_FLAG_PREDICTOR = 4      /* the handle also holds a [max_batch][n][R] buffer for zl_predict_select_batched */
+    ZL_FLAG_PREDICTOR = 4,     /* the handle also holds a [max_batch][n][R] buffer for zl_predict_select_batched */
+    ZL_FLAG_DEBUG_CHECKS = 8   /* kernels test every computed index against its buffer before using it and record the
+                                  first violation instead of making the access (see zl_debug_report in zipline_debug.h) */
 };
 
 typedef struct {

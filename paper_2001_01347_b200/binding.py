@@ -16,7 +16,7 @@ from . import build as _build
 ZL_OK = 0
 ZL_ERR_INVALID_ARG, ZL_ERR_UNSUPPORTED, ZL_ERR_NOMEM, ZL_ERR_CUDA, ZL_ERR_UNSORTED, ZL_ERR_TIMEOUT = range(1, 7)
 ZL_OBJ_RANGE, ZL_OBJ_SUM = 0, 1
-ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP, ZL_FLAG_PREDICTOR = 1, 2, 4
+ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP, ZL_FLAG_PREDICTOR, ZL_FLAG_DEBUG_CHECKS = 1, 2, 4, 8
 
 EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace_batched", "zl_destroy",
            "zl_set_option", "zl_status_string", "zl_workspace_bytes", "zl_launches_per_call",
@@ -24,7 +24,7 @@ EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace
            "zl_profile_begin", "zl_profile_read", "zl_profile_end",
            "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes", "zl_filter_counts",
            "zl_predict_batched", "zl_predict_select_batched", "zl_gridscan_batched", "zl_route",
-           "zl_probe_read_batched")
+           "zl_probe_read_batched", "zl_debug_report", "zl_debug_stamps", "zl_uses_cluster_kernel")
 
 
 class zl_config(ctypes.Structure):
@@ -63,6 +63,12 @@ def _load() -> ctypes.CDLL:
     lib.zl_predict_select_batched.restype = ctypes.c_int
     lib.zl_filter_counts.argtypes = [vp, i32, vp, vp, vp]
     lib.zl_filter_counts.restype = ctypes.c_int
+    lib.zl_debug_report.argtypes = [vp, vp]
+    lib.zl_debug_report.restype = ctypes.c_int
+    lib.zl_uses_cluster_kernel.argtypes = [vp]
+    lib.zl_debug_stamps.argtypes = [vp, i32, vp]
+    lib.zl_debug_stamps.restype = ctypes.c_int
+    lib.zl_uses_cluster_kernel.restype = ctypes.c_int
     lib.zl_select_batched_noalloc.argtypes = [i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
     lib.zl_select_batched_noalloc.restype = ctypes.c_int
     lib.zl_noalloc_max_batch.restype = ctypes.c_int
@@ -205,6 +211,24 @@ class ZipLine:
         _check(lib.zl_filter_counts(self._h, B, ctypes.addressof(f), ctypes.addressof(r), ctypes.addressof(o)),
                "zl_filter_counts")
         return list(f), list(r), list(o)
+
+    def debug_report(self):
+        """(code, cta, index) of the first index violation since the last report, (0, 0, 0) if none.  Synchronises."""
+        rec = (ctypes.c_uint32 * 4)()
+        _check(lib.zl_debug_report(self._h, ctypes.addressof(rec)), "zl_debug_report")
+        return int(rec[0]), int(rec[1]), int(rec[2]) | (int(rec[3]) << 32)
+
+    def debug_stamps(self, ctas: int):
+        """[ctas, 16] uint64 nanosecond stamps of the cluster kernel's phase boundaries in the last call (numpy)."""
+        import numpy as np
+        out = np.zeros((ctas, 16), dtype=np.uint64)
+        _check(lib.zl_debug_stamps(self._h, ctas, out.ctypes.data), "zl_debug_stamps")
+        return out
+
+    @property
+    def uses_cluster_kernel(self) -> bool:
+        """True when the handle's calls run the RANGE filter route as one cluster kernel."""
+        return bool(lib.zl_uses_cluster_kernel(self._h))
 
     def set_option(self, key: str, value: int):
         _check(lib.zl_set_option(self._h, key.encode(), int(value)), f"zl_set_option({key})")

@@ -43,7 +43,8 @@ struct zl_handle {
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round, opt_no_fused, opt_cluster, opt_filter_stages, opt_prefetch_rows, opt_checks_off;
+    int epoch;               // calls so far: the two sets of per-call flags alternate
     int last_cuda_error;
     int launches;
     // optional per-kernel timing: PROF_EVENTS events per recorded call
@@ -70,9 +71,14 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     zl::FilterBufs fb = q.fb;
     if (!filter && !sumfast) memset(&fb, 0, sizeof(fb));
     if (ev) cudaEventRecord(ev[0], st);
-    zl::enqueue_prologue(q, fb, st, src);
+    const bool fused = filter && q.fused;
+    if (!fused) zl::enqueue_prologue(q, fb, st, src);
     if (ev) cudaEventRecord(ev[1], st);
-    if (filter) {
+    if (fused) {
+        zl::enqueue_fused(q, fb, st, src);
+        if (ev) cudaEventRecord(ev[2], st);
+        zl::enqueue_heavy(q, fb, st);
+    } else if (filter) {
         zl::enqueue_filter(q, fb, st, ev ? ev[2] : nullptr, src);
         zl::enqueue_heavy(q, fb, st);
     } else if (sumfast) {
@@ -89,6 +95,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
 cudaError_t raise_shared_memory_limits() {
     cudaError_t e = zl::prologue_limits();
     if (e == cudaSuccess) e = zl::filter_limits();
+    if (e == cudaSuccess) e = zl::fused_limits();
     if (e == cudaSuccess) e = zl::heavy_limits();
     if (e == cudaSuccess) e = zl::bucket_route_limits();
     if (e == cudaSuccess) e = zl::sweep_limits();
@@ -157,7 +164,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     *out = nullptr;
     if (cfg->n_workers < 1 || cfg->lookahead_R < 1 || cfg->max_batch < 1) return ZL_ERR_INVALID_ARG;
     if (cfg->objective != ZL_OBJ_RANGE && cfg->objective != ZL_OBJ_SUM) return ZL_ERR_INVALID_ARG;
-    if (cfg->flags & ~(ZL_FLAG_CHECK_SORTED | ZL_FLAG_FULL_SWEEP | ZL_FLAG_PREDICTOR)) return ZL_ERR_INVALID_ARG;
+    if (cfg->flags & ~(ZL_FLAG_CHECK_SORTED | ZL_FLAG_FULL_SWEEP | ZL_FLAG_PREDICTOR | ZL_FLAG_DEBUG_CHECKS)) return ZL_ERR_INVALID_ARG;
     if (cfg->n_workers > zl::MAX_WORKERS) return ZL_ERR_UNSUPPORTED;
     if ((long long)cfg->n_workers * cfg->lookahead_R > (1LL << 31) - 1) return ZL_ERR_UNSUPPORTED;
     if (cfg->max_batch > 65535) return ZL_ERR_UNSUPPORTED;
@@ -189,13 +196,26 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         f.list1cap = (int)(N <= (1 << 17) ? N : N / 2);            // small shapes: room for every element
         h->nres = std::max(zl::MAX_SEGMENTS, (f.nbk + f.grp - 1) / f.grp);
         const size_t tiles = ((size_t)f.fcells + zl::SCAN_TILE - 1) / zl::SCAN_TILE;
-        const size_t sizes[9] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.fcells * 4, mb * cfg->n_workers * 4,
-                                 mb * (size_t)f.list1cap * 8, mb * f.nbk * 4, mb * f.nbk * f.capb * 8, mb * tiles * 4, 64};
-        void **ptrs[9] = {(void **)&f.table, (void **)&f.rowhint, (void **)&f.cellmax, (void **)&f.rcnt,
-                          (void **)&f.list1, (void **)&f.bcnt, (void **)&f.list2, (void **)&f.tilemax, (void **)&f.flags};
-        for (int i = 0; i < 9; ++i) {
+        // the fused kernel runs up to max(max_batch, 8 x SMs) CTAs, each with a record of partial results and a partial table
+        const size_t ctas = std::max<size_t>(mb, (size_t)h->num_sms * 8);
+        const size_t sizes[11] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.fcells * 4, std::max<size_t>(mb * cfg->n_workers, ctas) * 4,
+                                  mb * (size_t)f.list1cap * 8, mb * f.nbk * 4, mb * f.nbk * f.capb * 8, mb * tiles * 4, 64,
+                                  ctas * 4 * 8, ctas * f.cells * 4};
+        void **ptrs[11] = {(void **)&f.table, (void **)&f.rowhint, (void **)&f.cellmax, (void **)&f.rcnt,
+                           (void **)&f.list1, (void **)&f.bcnt, (void **)&f.list2, (void **)&f.tilemax, (void **)&f.flags,
+                           (void **)&f.part, (void **)&f.ptab};
+        f.maxctas = (int)std::min<size_t>(ctas, 0x7fffffff);
+        for (int i = 0; i < 11; ++i) {
             if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
             filter_b += sizes[i];
+        }
+        if (e == cudaSuccess) e = cudaMemset(f.flags, 0, 64);
+        if (cfg->flags & ZL_FLAG_DEBUG_CHECKS) {
+            // the violation record, then 16 clock stamps per CTA of the cluster kernel
+            const size_t dbg_b = 64 + ctas * 16 * 8;
+            if (e == cudaSuccess) e = cudaMalloc((void **)&f.dbg, dbg_b);
+            if (e == cudaSuccess) e = cudaMemset(f.dbg, 0, dbg_b);
+            filter_b += dbg_b;
         }
     }
     if (cfg->objective == ZL_OBJ_SUM || range_small) {
@@ -221,6 +241,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
                 if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
                 filter_b += sizes[i];
             }
+            if (e == cudaSuccess) e = cudaMemset(f.flags, 0, 64);
             h->nres = std::max(zl::MAX_SEGMENTS, f.stiles * zl::TILE_BK);   // up to one result per bucket
         } else {
             memset(&f, 0, sizeof(f));
@@ -237,7 +258,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
         cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
         cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
-        cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab);
+        cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab); cudaFree(h->fb.part); cudaFree(h->fb.ptab); cudaFree(h->fb.dbg);
         delete h;
         return st;
     }
@@ -300,7 +321,7 @@ zl_status zl_destroy(zl_handle *h) {
     cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
     cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
     cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
-    cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab);
+    cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab); cudaFree(h->fb.part); cudaFree(h->fb.ptab); cudaFree(h->fb.dbg);
     cudaFree(h->s_ts); cudaFree(h->s_idx); cudaFree(h->s_barrier); cudaFree(h->s_wait); cudaFree(h->s_status);
     if (h->s_stream) cudaStreamDestroy(h->s_stream);
     zl_profile_end(h);
@@ -322,6 +343,19 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
         h->opt_segments = value;
     } else if (!strcmp(key, "no_filter")) {
         h->opt_no_filter = value != 0;
+    } else if (!strcmp(key, "no_fused")) {
+        h->opt_no_fused = value != 0;
+    } else if (!strcmp(key, "cluster")) {
+        if (value > 8) return ZL_ERR_INVALID_ARG;
+        h->opt_cluster = value;
+    } else if (!strcmp(key, "filter_stages")) {
+        if (value && (value < 2 || value > 8)) return ZL_ERR_INVALID_ARG;
+        h->opt_filter_stages = value;
+    } else if (!strcmp(key, "prefetch_rows")) {
+        if (value > 32) return ZL_ERR_INVALID_ARG;
+        h->opt_prefetch_rows = value;
+    } else if (!strcmp(key, "checks_off")) {
+        h->opt_checks_off = value != 0;             // a ZL_FLAG_DEBUG_CHECKS handle keeps its clock stamps but runs the unchecked kernels
     } else if (!strcmp(key, "filter_threads")) {
         if (value && (!is_pow2(value) || value < 64 || value > 1024)) return ZL_ERR_INVALID_ARG;
         h->opt_filter_threads = value;
@@ -350,7 +384,12 @@ int32_t zl_launches_per_call(const zl_handle *h) {
     if (!h) return 0;
     const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter && h->fb.table != nullptr;
     const bool sumfast = !filter && !h->opt_no_filter && h->fb.scap != 0;
-    return 3 + (filter ? 6 : 0) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
+    const bool fused = filter && !h->opt_no_fused && !(h->cfg.flags & ZL_FLAG_CHECK_SORTED);
+    return (fused ? 7 : 3 + (filter ? 6 : 0)) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
+}
+int32_t zl_uses_cluster_kernel(const zl_handle *h) {
+    return h && !h->opt_no_filter && !h->opt_no_fused && h->cfg.objective == ZL_OBJ_RANGE && h->fb.table != nullptr &&
+           !(h->cfg.flags & ZL_FLAG_CHECK_SORTED);
 }
 int32_t zl_route(const zl_handle *h) {
     if (!h || h->opt_no_filter) return 0;
@@ -380,11 +419,40 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.filter_round = h->opt_filter_round; q.pdl_off = h->opt_pdl_off;
     q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
     if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
+    q.fused = !h->opt_no_fused && !(q.flags & ZL_FLAG_CHECK_SORTED);
+    q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
+    q.prefetch_rows = h->opt_prefetch_rows; q.checks_off = h->opt_checks_off;
+    if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
+        uint32_t *base = h->fb.flags;
+        q.fb.flags = base + 8 * (h->epoch & 1);
+        q.fb.flags_next = base + 8 * ((h->epoch + 1) & 1);
+        ++h->epoch;
+    }
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, st, ev, zl::MatBatch{d_ts});
     if (ev) ++h->prof_calls;
     ZL_CUDA(h, cudaGetLastError());
     h->launches += zl_launches_per_call(h);
+    return ZL_OK;
+}
+
+zl_status zl_debug_stamps(zl_handle *h, int32_t ctas, uint64_t *h_stamps) {
+    if (!h || !h_stamps || ctas < 1) return ZL_ERR_INVALID_ARG;
+    if (!h->fb.dbg || ctas > h->fb.maxctas) return ZL_ERR_INVALID_ARG;
+    ZL_CUDA(h, cudaSetDevice(h->cfg.device));
+    ZL_CUDA(h, cudaDeviceSynchronize());
+    ZL_CUDA(h, cudaMemcpy(h_stamps, h->fb.dbg + 16, (size_t)ctas * 16 * 8, cudaMemcpyDeviceToHost));
+    return ZL_OK;
+}
+
+zl_status zl_debug_report(zl_handle *h, uint32_t *h_record) {
+    if (!h || !h_record) return ZL_ERR_INVALID_ARG;
+    memset(h_record, 0, 4 * sizeof(uint32_t));
+    if (!h->fb.dbg) return ZL_OK;
+    ZL_CUDA(h, cudaSetDevice(h->cfg.device));
+    ZL_CUDA(h, cudaDeviceSynchronize());
+    ZL_CUDA(h, cudaMemcpy(h_record, h->fb.dbg, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost));
+    ZL_CUDA(h, cudaMemset(h->fb.dbg, 0, 4 * sizeof(uint32_t)));
     return ZL_OK;
 }
 
@@ -423,6 +491,15 @@ zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const i
         q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.filter_round = h->opt_filter_round; q.pdl_off = h->opt_pdl_off;
         q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
         if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
+        q.fused = !h->opt_no_fused && !(q.flags & ZL_FLAG_CHECK_SORTED);
+        q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
+        q.prefetch_rows = h->opt_prefetch_rows; q.checks_off = h->opt_checks_off;
+        if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
+            uint32_t *base = h->fb.flags;
+            q.fb.flags = base + 8 * (h->epoch & 1);
+            q.fb.flags_next = base + 8 * ((h->epoch + 1) & 1);
+            ++h->epoch;
+        }
         q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
         enqueue(q, p, (cudaStream_t)cuda_stream, ev, zl::AriBatch{d_last, d_interval});
         if (ev) ++h->prof_calls;
@@ -541,7 +618,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
     q.meta = meta; q.seg = seg; q.nres = p.nseg;
     memset(&q.fb, 0, sizeof(q.fb));
-    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0;
+    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0; q.fused = 0; q.cluster = q.filter_stages = q.prefetch_rows = 0; q.checks_off = 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr, zl::MatBatch{d_ts});
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;

@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(1024, 1) k_prologue(const SRC src, int n, int 
     }
     __syncthreads();
     const InstMeta M = sm;
-    if (b == 0 && tid < 3 && F.flags) F.flags[tid] = 0;
+    if (b == 0 && tid < 3 && F.flags) { F.flags[tid] = 0; if (F.flags_next) F.flags_next[tid] = 0; }
     if (M.cscale != 0) {
         const uint32_t cells = (uint32_t)F.cells, cscale = M.cscale, lmin = (uint32_t)M.lmin;
         const uint32_t wcell = 0xffffffffu / cscale + 2;          // > 2^32 / cscale

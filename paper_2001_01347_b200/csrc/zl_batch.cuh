@@ -114,8 +114,16 @@ __device__ inline void block_best_to_result(uint64_t bd, uint64_t bt, uint32_t s
 // loaded together, then the seven elements between the two probes that bracket bar, loaded together: three
 // rounds of loads in the usual case.  A guess that is further off is bracketed by doubling steps and bisected.
 template <class ROW>
+__device__ int last_index_not_after(const ROW &row, int R, int64_t bar, int64_t e0, int64_t eR);
+
+template <class ROW>
 __device__ int last_index_not_after(const ROW &row, int R, int64_t bar) {
-    const int64_t e0 = row.at(0), eR = row.at(R - 1);
+    return last_index_not_after(row, R, bar, row.at(0), row.at(R - 1));
+}
+
+// The same with the row's first and last element already at hand.
+template <class ROW>
+__device__ int last_index_not_after(const ROW &row, int R, int64_t bar, int64_t e0, int64_t eR) {
     if (bar < e0) return -1;
     if (bar >= eR) return R - 1;
     // e0 <= bar < eR, R >= 2.  Invariant: row[lo - 1] <= bar, row[hi] > bar

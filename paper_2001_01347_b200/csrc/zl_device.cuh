@@ -210,4 +210,43 @@ __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.w
 
 __device__ __forceinline__ int64_t ldg64(const int64_t *p) { return (int64_t)__ldg((const long long *)p); }
 
+// ---------------------------------------------------------------------------------- bulk copies
+// One thread asks the copy engine for a contiguous piece of global memory; the bytes land in shared memory
+// and are counted on an mbarrier, whose phase completes when the announced number has arrived.  Both
+// addresses and the size are multiples of 16 bytes.  No multicast: the destination is the CTA's own memory.
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t *bar, int arrivals) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(arrivals) : "memory");
+}
+// An mbarrier has to be invalidated before its bytes serve any other purpose (or are initialised again).
+__device__ __forceinline__ void mbar_inval(uint64_t *bar) {
+    asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_copy_g2s(void *dst, const void *src, uint32_t bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+// shared-memory reads through ordinary loads come before later writes of the copy engine to the same bytes
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Wait for the phase with the given parity; gives up after a bounded number of polls (each poll may itself be
+// suspended by the hardware for a while) and reports it, so that a copy that never lands cannot hang the GPU.
+constexpr int MBAR_POLL_LIMIT = 1 << 22;
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity) {
+    for (int spins = 0; spins < MBAR_POLL_LIMIT; ++spins)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ uint32_t ldcg32(const uint32_t *p) { return __ldcg(p); }
+__device__ __forceinline__ uint64_t ldcg64(const uint64_t *p) { return (uint64_t)__ldcg((const unsigned long long *)p); }
+
 }  // namespace zl

@@ -25,6 +25,9 @@ struct Pipeline {
     int filter_threads, filter_rows, filter_round;                // 0: automatic
     int pdl_off;                                                  // bit mask of kernels launched without early scheduling
     int prologue_threads, tail_threads;                           // 0: automatic
+    int fused;                                                    // RANGE filter route: one cluster launch instead of prologue, filter pass and tail
+    int cluster, filter_stages, prefetch_rows;                    // of the cluster kernel; 0: automatic
+    int checks_off;                                               // debug handle: unchecked kernels, clock stamps still taken
     int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;
 };
 
@@ -57,6 +60,13 @@ cudaError_t prologue_limits();
 void enqueue_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid, const MatBatch &src);
 void enqueue_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid, const AriBatch &src);
 cudaError_t filter_limits();
+
+// fused.cu: the RANGE filter route of an instance by one thread-block cluster in one launch (column scans, filter
+// table, filter pass, finish of instances with few survivors, index recovery)
+cudaError_t enqueue_fused(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const MatBatch &src);
+cudaError_t enqueue_fused(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const AriBatch &src);
+int fused_cluster_size(int B, int n, int num_sms, int gmax);
+cudaError_t fused_limits();
 
 // heavy.cu: RANGE instances with many survivors (cell scan, refinement, bucket sweep)
 void enqueue_heavy(const Pipeline &q, const FilterBufs &fb, cudaStream_t st);

@@ -89,6 +89,11 @@ struct FilterBufs {
     uint32_t *rcnt;      // [B][nreg]         survivors per region (one region per CTA of the filter pass)
     uint64_t *list1;     // [B][list1cap]     survivors of the filter pass as (T << 32 | next), by region
     uint32_t *flags;     // [3]               per call: some instance needs [0] scan/refine/buckets, [1] the segment sweep, [2] k_finalize
+    uint32_t *flags_next; // [3]              the flags of the handle's next call (the two sets alternate); zeroed by this call
+    uint64_t *part;      // [ctas][4]         fused kernel: per-CTA minima / maxima of the first and last column
+    uint32_t *ptab;      // [ctas][cells]     fused kernel: per-CTA partial filter tables
+    int32_t maxctas;     //                   CTAs the fused kernel's per-CTA records have room for
+    uint32_t *dbg;       // [4]               ZL_FLAG_DEBUG_CHECKS: record of the first index violation (0: none)
     uint32_t *bcnt;      // [B][nbk]          survivors of the refinement per bucket
     uint64_t *list2;     // [B][nbk][capb]    survivors of the refinement
     int32_t cells, fcells, nbk, capb, grp;   // grp: fewest buckets per CTA of the bucket sweep
