@@ -176,11 +176,10 @@ def run_reference(args, w, objective):
     print(json.dumps(line), flush=True)
 
 
-STAGES = {  # names of what runs between the library's stage events, by (route, cluster kernel)
-    (1, True): ("-", "k_range_fused", "k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep", "k_finalize"),
-    (1, False): ("k_prologue", "k_filter", "k_tail+k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep", "k_finalize"),
-    (2, False): ("k_prologue", "k_sum_plan+k_sum_index", "k_sum_buckets+k_sweep", "k_finalize"),
-    (0, False): ("k_prologue", "-", "k_sweep", "k_finalize"),
+STAGES = {  # names of what runs between the library's stage events, by route
+    1: ("k_range_head", "k_range_filter", "k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep", "k_finalize"),
+    2: ("k_prologue", "k_sum_plan+k_sum_index", "k_sum_buckets+k_sweep", "k_finalize"),
+    0: ("k_prologue", "-", "k_sweep", "k_finalize"),
 }
 
 
@@ -234,7 +233,6 @@ def main():
 
     h = make_handle(0)
     route = h.route                                  # 0 segment sweep only, 1 RANGE filter route, 2 bucket route
-    cluster = bool(h.uses_cluster_kernel)
     examined = examined_early if route == 1 else nts
     copies = max(1, min(16, int(np.ceil(300e6 / (examined * 8)))))
     d_ts = [torch.from_numpy(ts_np).to(dev)]
@@ -359,7 +357,7 @@ def main():
 
     # ---- roofline of the dominant kernel: algorithmic bytes = 8 per timestamp it must examine
     peak, peak_kind = measured_peak_gbs()
-    names = STAGES[(route, cluster)]
+    names = STAGES[route]
 
     def dominant(pr):
         stages = dict(zip(names, (pr["ms_prologue"], pr["ms_filter"], pr["ms_sweep"], pr["ms_finalize"])))
@@ -398,7 +396,7 @@ def main():
                "sample": f"the first {inst} of {w.B} instances of {w.name}, sweep_window (sort + one pass), {dt:.1f} s wall"}
 
     result = {"selections_per_s": world * w.B / (ms_step * 1e-3), "early_stop": route == 1,
-              "route": {0: "segment sweep", 1: "filter", 2: "buckets"}[route], "cluster_kernel": cluster,
+              "route": {0: "segment sweep", 1: "filter", 2: "buckets"}[route],
               "examined_fraction": examined / nts, "input_copies": copies,
               "value_counts": "all n*R*B timestamps of the batch per call (nominal: the early stop examines examined_fraction of them; "
                               "full_sweep.value counts examined timestamps only)",

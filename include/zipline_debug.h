@@ -59,28 +59,25 @@ zl_status zl_filter_counts(zl_handle *h, int32_t B, uint32_t *h_filtered, uint32
  * copy, is compared with the extent of its buffer first; an index out of range is not used (the access is
  * skipped, nothing traps) and the first such event is recorded.  zl_debug_report waits for the device, copies the
  * record to h_record[0..3] (host) and clears it: [0] a code naming the access (0: no violation since the last
- * report), [1] the CTA, [2], [3] the low and high word of the offending index.  Covers the cluster kernel of the
- * RANGE filter route.
+ * report), [1] the CTA, [2], [3] the low and high word of the offending index.  Covers the two kernels of
+ * the RANGE filter route (k_range_head, k_range_filter).
  */
 zl_status zl_debug_report(zl_handle *h, uint32_t *h_record);
 
 /*
- * With the same flag the cluster kernel also notes the GPU's nanosecond clock at its phase boundaries: for each
- * of the first `ctas` CTAs of the handle's last call, 16 values (0 where a boundary was not passed) - start,
- * columns done, summary, partial table done, tables merged, filter pass begins, filter pass done, lists complete,
- * instance finished, result known, indices done.  h_stamps: host, ctas * 16 uint64.  Synchronises.
+ * With the same flag k_range_head also notes the GPU's nanosecond clock at its phase boundaries: for each of the
+ * first `ctas` CTAs of the handle's last call, 16 values (0 where a boundary was not passed): [0] start, [1] columns
+ * done, [2] summary, [11] requests written, [12] slow rows walked, [13] partial table done, [3] before and [4] after
+ * the cluster barrier, [5] merged table written.  h_stamps: host, ctas * 16 uint64.  Synchronises.
  */
 zl_status zl_debug_stamps(zl_handle *h, int32_t ctas, uint64_t *h_stamps);
-
-/* 1 when the handle's calls run the RANGE filter route as one cluster kernel (fused.cu), else 0. */
-int32_t zl_uses_cluster_kernel(const zl_handle *h);
 
 /* Tuning knobs of a handle (host side; take effect at the next call).
  * key: "threads" (128..1024, power of two), "lanes_per_row" (1..32, power of two),
  * "segments" (time segments per instance, >= 1), "round_factor" (percent of the
  * nominal elements per round), "no_filter" (1: neither the RANGE filter route nor the bucket
  * route is used; every instance is swept by time segments), "filter_threads" / "filter_rows" (CTA size and rows per CTA of the
- * filter pass), "no_fused" (1: the RANGE filter route runs as separate prologue, filter and tail kernels instead of one cluster kernel), "cluster" (CTAs per instance of the cluster kernel, a power of two up to 8), "filter_stages" (ring slots per warp, 2..8), "prefetch_rows" (rows per warp whose start is prefetched into the L2 at kernel start; default none), "checks_off" (1: a handle created with ZL_FLAG_DEBUG_CHECKS runs the unchecked kernels but still records the clock stamps), "filter_round" (a row is requested up to its estimate rounded up to this many timestamps; power of two, 2..256), "prologue_threads" / "tail_threads" (CTA sizes of those kernels), "pdl_off" (bit k: launch the k-th kernel of the chain only after its predecessor has
+ * filter pass), "cluster" (CTAs per instance of the first kernel of the RANGE filter route, a power of two up to 8), "filter_stages" (ring slots per warp, 2..7), "filter_bulk" (1: chunks of a row arrive by one bulk-copy request each, 2: in 16-byte pieces copied by every lane; default: bulk requests for whole rows, pieces for the prefixes of the early stop), "checks_off" (1: a handle created with ZL_FLAG_DEBUG_CHECKS runs the unchecked kernels but still records the clock stamps), "filter_round" (a row is requested up to its estimate rounded up to this many timestamps; power of two, 2..1024; from 128 on it is also the ring slot size of the cluster kernel), "prologue_threads" / "tail_threads" (CTA sizes of those kernels), "pdl_off" (bit k: launch the k-th kernel of the chain only after its predecessor has
  * finished instead of scheduling it early).  0 restores the built-in choice. */
 zl_status zl_set_option(zl_handle *h, const char *key, int32_t value);
 

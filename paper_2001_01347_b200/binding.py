@@ -24,7 +24,7 @@ EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace
            "zl_profile_begin", "zl_profile_read", "zl_profile_end",
            "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes", "zl_filter_counts",
            "zl_predict_batched", "zl_predict_select_batched", "zl_gridscan_batched", "zl_route",
-           "zl_probe_read_batched", "zl_debug_report", "zl_debug_stamps", "zl_uses_cluster_kernel")
+           "zl_probe_read_batched", "zl_debug_report", "zl_debug_stamps")
 
 
 class zl_config(ctypes.Structure):
@@ -65,10 +65,8 @@ def _load() -> ctypes.CDLL:
     lib.zl_filter_counts.restype = ctypes.c_int
     lib.zl_debug_report.argtypes = [vp, vp]
     lib.zl_debug_report.restype = ctypes.c_int
-    lib.zl_uses_cluster_kernel.argtypes = [vp]
     lib.zl_debug_stamps.argtypes = [vp, i32, vp]
     lib.zl_debug_stamps.restype = ctypes.c_int
-    lib.zl_uses_cluster_kernel.restype = ctypes.c_int
     lib.zl_select_batched_noalloc.argtypes = [i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, vp]
     lib.zl_select_batched_noalloc.restype = ctypes.c_int
     lib.zl_noalloc_max_batch.restype = ctypes.c_int
@@ -224,11 +222,6 @@ class ZipLine:
         out = np.zeros((ctas, 16), dtype=np.uint64)
         _check(lib.zl_debug_stamps(self._h, ctas, out.ctypes.data), "zl_debug_stamps")
         return out
-
-    @property
-    def uses_cluster_kernel(self) -> bool:
-        """True when the handle's calls run the RANGE filter route as one cluster kernel."""
-        return bool(lib.zl_uses_cluster_kernel(self._h))
 
     def set_option(self, key: str, value: int):
         _check(lib.zl_set_option(self._h, key.encode(), int(value)), f"zl_set_option({key})")

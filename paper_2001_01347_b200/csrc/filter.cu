@@ -1,5 +1,6 @@
 // The RANGE filter pass (k_filter on stored rows, k_filter_arith on predicted rows) and k_tail, which finishes
-// the instances that are left with few survivors.
+// the instances that are left with few survivors: the kernels every handle runs unless it asks for the checked
+// ones (range_filter.cu).
 #include "zl_batch.cuh"
 #include "zl_host.h"
 
@@ -14,27 +15,6 @@ namespace zl {
 constexpr int FILTER_STAGES = 3;      // ring slots per warp
 constexpr int FILTER_CHUNK = 256;     // timestamps per slot (FILTER_CHUNK / 64 16-byte copies per lane)
 constexpr int FILTER_SLOT = FILTER_CHUNK + 2;   // + the successor of the slot's last element, + padding
-
-__device__ __forceinline__ void cp_async16(void *smem, const void *gmem) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
-}
-__device__ __forceinline__ void cp_async8(void *smem, const void *gmem) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;\n" ::"r"((uint32_t)__cvta_generic_to_shared(smem)), "l"(gmem) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-// wait until at most `pending` of this thread's most recent groups are still in flight
-__device__ __forceinline__ void cp_async_wait_pending(int pending) {
-    switch (pending) {
-        case 0: asm volatile("cp.async.wait_group 0;\n" ::: "memory"); break;
-        case 1: asm volatile("cp.async.wait_group 1;\n" ::: "memory"); break;
-        case 2: asm volatile("cp.async.wait_group 2;\n" ::: "memory"); break;
-        case 3: asm volatile("cp.async.wait_group 3;\n" ::: "memory"); break;
-        case 4: asm volatile("cp.async.wait_group 4;\n" ::: "memory"); break;
-        case 5: asm volatile("cp.async.wait_group 5;\n" ::: "memory"); break;
-        case 6: asm volatile("cp.async.wait_group 6;\n" ::: "memory"); break;
-        default: asm volatile("cp.async.wait_group 7;\n" ::: "memory"); break;
-    }
-}
 
 struct FilterCtx {
     const uint32_t *tab; uint64_t *list; uint32_t *cellmax; unsigned int *scount;

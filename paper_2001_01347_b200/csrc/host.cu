@@ -43,7 +43,7 @@ struct zl_handle {
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round, opt_no_fused, opt_cluster, opt_filter_stages, opt_prefetch_rows, opt_checks_off;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round, opt_cluster, opt_filter_stages, opt_checks_off, opt_filter_bulk, opt_tail_cap;
     int epoch;               // calls so far: the two sets of per-call flags alternate
     int last_cuda_error;
     int launches;
@@ -62,6 +62,10 @@ constexpr int PROF_EVENTS = 5;
 
 // SRC: zl::MatBatch (the rows are read from q.ts) or zl::AriBatch (predicted rows, generated on the fly; RANGE, filter
 // route or plain segment sweep only).
+// RANGE filter route: from this many timestamps an instance on, what the filter and tail kernels leave undone goes
+// through kernels of its own per phase instead of the single last kernel.
+static bool range_rest_split(int n, int R) { return (long long)n * R >= (1LL << 21); }
+
 template <class SRC>
 void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_t *ev, const SRC src) {
     constexpr bool arith = std::is_same<SRC, zl::AriBatch>::value;
@@ -71,15 +75,29 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     zl::FilterBufs fb = q.fb;
     if (!filter && !sumfast) memset(&fb, 0, sizeof(fb));
     if (ev) cudaEventRecord(ev[0], st);
-    const bool fused = filter && q.fused;
-    if (!fused) zl::enqueue_prologue(q, fb, st, src);
+    if (filter) zl::enqueue_range_head(q, fb, st, src);
+    else zl::enqueue_prologue(q, fb, st, src);
+    if constexpr (!arith) if (q.flags & ZL_FLAG_CHECK_SORTED) zl::enqueue_check_sorted(q, st);
     if (ev) cudaEventRecord(ev[1], st);
-    if (fused) {
-        zl::enqueue_fused(q, fb, st, src);
-        if (ev) cudaEventRecord(ev[2], st);
-        zl::enqueue_heavy(q, fb, st);
-    } else if (filter) {
-        zl::enqueue_filter(q, fb, st, ev ? ev[2] : nullptr, src);
+    if (filter) {
+        // the filter kernel, then everything it left undone and the outputs in one more launch
+        const bool checked = ((q.flags & ZL_FLAG_DEBUG_CHECKS) && !q.checks_off) || q.filter_bulk;
+        if (checked) {
+            // the self-checking variants of the two kernels (also the ones with the bulk-copy ring)
+            zl::enqueue_range_filter(q, fb, st, src);
+            if (ev) cudaEventRecord(ev[2], st);
+            zl::enqueue_range_tail(q, fb, st, src);
+        } else {
+            zl::enqueue_filter(q, fb, st, ev ? ev[2] : nullptr, src);
+        }
+        if (ev) cudaEventRecord(ev[3], st);
+        if (!range_rest_split(q.n, q.R)) {
+            // everything the two kernels left undone, and the outputs, in one more launch
+            zl::enqueue_range_rest(q, fb, p, st, src);
+            if (ev) cudaEventRecord(ev[4], st);
+            return;
+        }
+        // large instances: survivors by the million are the rule, every phase gets a grid of its own
         zl::enqueue_heavy(q, fb, st);
     } else if (sumfast) {
         if constexpr (!arith) zl::enqueue_bucket_route(q, fb, st, ev ? ev[2] : nullptr);
@@ -94,9 +112,10 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
 
 cudaError_t raise_shared_memory_limits() {
     cudaError_t e = zl::prologue_limits();
+    if (e == cudaSuccess) e = zl::range_limits();
     if (e == cudaSuccess) e = zl::filter_limits();
-    if (e == cudaSuccess) e = zl::fused_limits();
     if (e == cudaSuccess) e = zl::heavy_limits();
+    if (e == cudaSuccess) e = zl::range_rest_limits();
     if (e == cudaSuccess) e = zl::bucket_route_limits();
     if (e == cudaSuccess) e = zl::sweep_limits();
     return e;
@@ -130,6 +149,10 @@ LaunchPlan make_plan(const zl_handle *h, int B) {
     target = std::min<long long>(target, (long long)p.cap * 4);
     p.target = (int)std::max<long long>(target, 32);
     p.smem = (((size_t)2 * n * sizeof(uint32_t) + 15) & ~(size_t)15) + (size_t)p.cap * 20;   // nodes, sorted nodes, slot counters
+    p.G_rest = h->opt_lanes ? std::min(h->opt_lanes, 512) : std::max(1, std::min(32, pow2_floor(std::max(1, 512 / n))));
+    long long target_rest = (long long)n * std::max(p.G_rest, 4) * rf / 100;
+    target_rest = std::min<long long>(target_rest, (long long)p.cap * 4);
+    p.target_rest = (int)std::max<long long>(target_rest, 32);
     return p;
 }
 
@@ -198,21 +221,21 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         const size_t tiles = ((size_t)f.fcells + zl::SCAN_TILE - 1) / zl::SCAN_TILE;
         // the fused kernel runs up to max(max_batch, 8 x SMs) CTAs, each with a record of partial results and a partial table
         const size_t ctas = std::max<size_t>(mb, (size_t)h->num_sms * 8);
-        const size_t sizes[11] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.fcells * 4, std::max<size_t>(mb * cfg->n_workers, ctas) * 4,
+        const size_t sizes[12] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.fcells * 4, std::max<size_t>(mb * cfg->n_workers, ctas) * 4,
                                   mb * (size_t)f.list1cap * 8, mb * f.nbk * 4, mb * f.nbk * f.capb * 8, mb * tiles * 4, 64,
-                                  ctas * 4 * 8, ctas * f.cells * 4};
-        void **ptrs[11] = {(void **)&f.table, (void **)&f.rowhint, (void **)&f.cellmax, (void **)&f.rcnt,
+                                  ctas * 4 * 8, ctas * f.cells * 4, mb * 4};
+        void **ptrs[12] = {(void **)&f.table, (void **)&f.rowhint, (void **)&f.cellmax, (void **)&f.rcnt,
                            (void **)&f.list1, (void **)&f.bcnt, (void **)&f.list2, (void **)&f.tilemax, (void **)&f.flags,
-                           (void **)&f.part, (void **)&f.ptab};
+                           (void **)&f.part, (void **)&f.ptab, (void **)&f.done};
         f.maxctas = (int)std::min<size_t>(ctas, 0x7fffffff);
-        for (int i = 0; i < 11; ++i) {
+        for (int i = 0; i < 12; ++i) {
             if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
             filter_b += sizes[i];
         }
         if (e == cudaSuccess) e = cudaMemset(f.flags, 0, 64);
         if (cfg->flags & ZL_FLAG_DEBUG_CHECKS) {
-            // the violation record, then 16 clock stamps per CTA of the cluster kernel
-            const size_t dbg_b = 64 + ctas * 16 * 8;
+            // the violation record, then 16 clock stamps per CTA of the head kernel and of the filter kernel
+            const size_t dbg_b = 64 + (ctas + mb * ((size_t)cfg->n_workers + 1) / 2 + 1) * 16 * 8;
             if (e == cudaSuccess) e = cudaMalloc((void **)&f.dbg, dbg_b);
             if (e == cudaSuccess) e = cudaMemset(f.dbg, 0, dbg_b);
             filter_b += dbg_b;
@@ -258,7 +281,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
         cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
         cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
-        cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab); cudaFree(h->fb.part); cudaFree(h->fb.ptab); cudaFree(h->fb.dbg);
+        cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab); cudaFree(h->fb.part); cudaFree(h->fb.ptab); cudaFree(h->fb.dbg); cudaFree(h->fb.done);
         delete h;
         return st;
     }
@@ -321,7 +344,7 @@ zl_status zl_destroy(zl_handle *h) {
     cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
     cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
     cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
-    cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab); cudaFree(h->fb.part); cudaFree(h->fb.ptab); cudaFree(h->fb.dbg);
+    cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab); cudaFree(h->fb.part); cudaFree(h->fb.ptab); cudaFree(h->fb.dbg); cudaFree(h->fb.done);
     cudaFree(h->s_ts); cudaFree(h->s_idx); cudaFree(h->s_barrier); cudaFree(h->s_wait); cudaFree(h->s_status);
     if (h->s_stream) cudaStreamDestroy(h->s_stream);
     zl_profile_end(h);
@@ -343,17 +366,18 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
         h->opt_segments = value;
     } else if (!strcmp(key, "no_filter")) {
         h->opt_no_filter = value != 0;
-    } else if (!strcmp(key, "no_fused")) {
-        h->opt_no_fused = value != 0;
     } else if (!strcmp(key, "cluster")) {
         if (value > 8) return ZL_ERR_INVALID_ARG;
         h->opt_cluster = value;
     } else if (!strcmp(key, "filter_stages")) {
-        if (value && (value < 2 || value > 8)) return ZL_ERR_INVALID_ARG;
+        if (value && (value < 2 || value > 7)) return ZL_ERR_INVALID_ARG;
         h->opt_filter_stages = value;
-    } else if (!strcmp(key, "prefetch_rows")) {
-        if (value > 32) return ZL_ERR_INVALID_ARG;
-        h->opt_prefetch_rows = value;
+    } else if (!strcmp(key, "filter_bulk")) {
+        if (value > 2) return ZL_ERR_INVALID_ARG;
+        h->opt_filter_bulk = value;
+    } else if (!strcmp(key, "tail_cap")) {
+        if (value != 0 && (value < 64 || value > 2048 || (value & (value - 1)))) return ZL_ERR_INVALID_ARG;
+        h->opt_tail_cap = (int)value;
     } else if (!strcmp(key, "checks_off")) {
         h->opt_checks_off = value != 0;             // a ZL_FLAG_DEBUG_CHECKS handle keeps its clock stamps but runs the unchecked kernels
     } else if (!strcmp(key, "filter_threads")) {
@@ -365,7 +389,7 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
     } else if (!strcmp(key, "pdl_off")) {
         h->opt_pdl_off = value;                 // bit k set: kernel k of the chain is launched without early scheduling
     } else if (!strcmp(key, "filter_round")) {
-        if (value && (!is_pow2(value) || value < 2 || value > 256)) return ZL_ERR_INVALID_ARG;
+        if (value && (!is_pow2(value) || value < 2 || value > 1024)) return ZL_ERR_INVALID_ARG;
         h->opt_filter_round = value;
     } else if (!strcmp(key, "filter_rows")) {
         if (value > 65536) return ZL_ERR_INVALID_ARG;
@@ -384,12 +408,7 @@ int32_t zl_launches_per_call(const zl_handle *h) {
     if (!h) return 0;
     const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter && h->fb.table != nullptr;
     const bool sumfast = !filter && !h->opt_no_filter && h->fb.scap != 0;
-    const bool fused = filter && !h->opt_no_fused && !(h->cfg.flags & ZL_FLAG_CHECK_SORTED);
-    return (fused ? 7 : 3 + (filter ? 6 : 0)) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
-}
-int32_t zl_uses_cluster_kernel(const zl_handle *h) {
-    return h && !h->opt_no_filter && !h->opt_no_fused && h->cfg.objective == ZL_OBJ_RANGE && h->fb.table != nullptr &&
-           !(h->cfg.flags & ZL_FLAG_CHECK_SORTED);
+    return (filter ? (range_rest_split(h->cfg.n_workers, h->cfg.lookahead_R) ? 9 : 4) : 3) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
 }
 int32_t zl_route(const zl_handle *h) {
     if (!h || h->opt_no_filter) return 0;
@@ -419,9 +438,8 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.filter_round = h->opt_filter_round; q.pdl_off = h->opt_pdl_off;
     q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
     if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
-    q.fused = !h->opt_no_fused && !(q.flags & ZL_FLAG_CHECK_SORTED);
     q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
-    q.prefetch_rows = h->opt_prefetch_rows; q.checks_off = h->opt_checks_off;
+    q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0;
     if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
         uint32_t *base = h->fb.flags;
         q.fb.flags = base + 8 * (h->epoch & 1);
@@ -438,7 +456,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
 
 zl_status zl_debug_stamps(zl_handle *h, int32_t ctas, uint64_t *h_stamps) {
     if (!h || !h_stamps || ctas < 1) return ZL_ERR_INVALID_ARG;
-    if (!h->fb.dbg || ctas > h->fb.maxctas) return ZL_ERR_INVALID_ARG;
+    if (!h->fb.dbg || ctas > (long long)h->fb.maxctas + ((long long)h->cfg.max_batch * (h->cfg.n_workers + 1)) / 2) return ZL_ERR_INVALID_ARG;
     ZL_CUDA(h, cudaSetDevice(h->cfg.device));
     ZL_CUDA(h, cudaDeviceSynchronize());
     ZL_CUDA(h, cudaMemcpy(h_stamps, h->fb.dbg + 16, (size_t)ctas * 16 * 8, cudaMemcpyDeviceToHost));
@@ -491,9 +509,8 @@ zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const i
         q.filter_threads = h->opt_filter_threads; q.filter_rows = h->opt_filter_rows; q.filter_round = h->opt_filter_round; q.pdl_off = h->opt_pdl_off;
         q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
         if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
-        q.fused = !h->opt_no_fused && !(q.flags & ZL_FLAG_CHECK_SORTED);
         q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
-        q.prefetch_rows = h->opt_prefetch_rows; q.checks_off = h->opt_checks_off;
+        q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0;
         if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
             uint32_t *base = h->fb.flags;
             q.fb.flags = base + 8 * (h->epoch & 1);
@@ -618,7 +635,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
     q.meta = meta; q.seg = seg; q.nres = p.nseg;
     memset(&q.fb, 0, sizeof(q.fb));
-    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0; q.fused = 0; q.cluster = q.filter_stages = q.prefetch_rows = 0; q.checks_off = 0;
+    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0; q.cluster = q.filter_stages = 0; q.checks_off = 0; q.filter_bulk = 0; q.tail_cap = 0; q.rest_per_sm = 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr, zl::MatBatch{d_ts});
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;

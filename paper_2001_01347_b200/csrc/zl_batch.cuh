@@ -110,9 +110,10 @@ __device__ inline void block_best_to_result(uint64_t bd, uint64_t bt, uint32_t s
 }
 
 // Index of the last element of a sorted row that is <= bar (-1 if none).  Rows are close to arithmetic, so the
-// position is first guessed from the row's end points.  Eight probes around the guess, eight elements apart and
-// loaded together, then the seven elements between the two probes that bracket bar, loaded together: three
-// rounds of loads in the usual case.  A guess that is further off is bracketed by doubling steps and bisected.
+// position is first guessed from the row's end points, and the sixteen consecutive elements around the guess are
+// loaded together (they share a cache line or two: the fewer distinct lines the call touches the better, since
+// every one of them is a memory access of its own).  A guess that is further off looks at the sixteen elements on
+// the side the answer lies on, twice at most, before it falls back to doubling steps and bisection.
 template <class ROW>
 __device__ int last_index_not_after(const ROW &row, int R, int64_t bar, int64_t e0, int64_t eR);
 
@@ -127,39 +128,32 @@ __device__ int last_index_not_after(const ROW &row, int R, int64_t bar, int64_t 
     if (bar < e0) return -1;
     if (bar >= eR) return R - 1;
     // e0 <= bar < eR, R >= 2.  Invariant: row[lo - 1] <= bar, row[hi] > bar
-    int lo, hi;
+    int lo = 1, hi = R - 1;
     int g = (int)((double)(bar - e0) * (double)(R - 1) / (double)(eR - e0));
     g = max(0, min(g, R - 2));
-    {
-        constexpr int S = 8, P = 8;                       // probes at g + S * (k - P/2), clamped to the row
-        int64_t pv[P];
-        int pi[P];
+    constexpr int W = 16;
+    int a = max(0, min(g - W / 2 + 1, R - W)) & ~3;                // the window [a, a + W), on a 32-byte boundary of the row
+    for (int it = 0; it < 3; ++it) {
+        int64_t v[W];
 #pragma unroll
-        for (int k = 0; k < P; ++k) { pi[k] = max(0, min(R - 1, g + S * (k - P / 2))); pv[k] = row.at(pi[k]); }
-        lo = 1; hi = R - 1;
+        for (int k = 0; k < W; ++k) v[k] = row.at(min(a + k, R - 1));
+        int c = 0, valid = 0;
 #pragma unroll
-        for (int k = 0; k < P; ++k) {
-            if (pv[k] <= bar) lo = max(lo, pi[k] + 1); else hi = min(hi, pi[k]);
-        }
-        if (hi - lo <= S - 1) {                            // bracketed between two neighbouring probes
-            int64_t wv[S - 1];
-#pragma unroll
-            for (int k = 0; k < S - 1; ++k) wv[k] = row.at(min(lo + k, R - 1));
-            int c = 0;
-#pragma unroll
-            for (int k = 0; k < S - 1; ++k) c += (lo + k < hi && wv[k] <= bar) ? 1 : 0;   // sorted: a prefix of the window
-            return lo + c - 1;
-        }
+        for (int k = 0; k < W; ++k) { valid += a + k < R ? 1 : 0; c += (a + k < R && v[k] <= bar) ? 1 : 0; }   // sorted: a prefix of the window
+        if (c > 0 && c < valid) return a + c - 1;                  // the window holds the last element <= bar and its successor
+        if (c == 0) hi = min(hi, a); else lo = max(lo, a + valid);
+        if (lo >= hi) return lo - 1;
+        a = c == 0 ? max(0, hi - W) : min(lo, max(0, R - W));
     }
-    // the probes did not enclose bar closely: doubling steps from the nearer end of the bracket, then bisection
-    if (lo > 1) {                                          // everything probed was <= bar: search upwards from lo
+    // the guess was far off: doubling steps from the nearer end of the bracket, then bisection
+    if (lo > 1) {                                          // everything looked at was <= bar: search upwards from lo
         const int top = hi;
         for (int step = 16; lo < hi; step <<= 1) {
             const int q = min(lo + step - 1, top - 1);
             if (q < lo) break;
             if (row.at(q) <= bar) lo = q + 1; else { hi = q; break; }
         }
-    } else {                                               // everything probed was > bar: search downwards from hi
+    } else {                                               // everything looked at was > bar: search downwards from hi
         for (int step = 16; lo < hi; step <<= 1) {
             const int q = max(hi - step, lo);
             if (row.at(q) > bar) hi = q; else { lo = q + 1; break; }
@@ -170,6 +164,62 @@ __device__ int last_index_not_after(const ROW &row, int R, int64_t bar, int64_t 
         if (row.at(mid) <= bar) lo = mid + 1; else hi = mid;
     }
     return lo - 1;
+}
+
+// The same for 32 stored rows at once, a row per lane (rowp == nullptr: the lane has none), by the whole warp: the
+// windows - 32 consecutive elements around each row's guess - are loaded a row an instruction (two or three lines
+// of memory, instead of one line per lane and element) and counted with a vote.  Rows whose answer three windows
+// do not find fall back to bisection.  Every lane of the warp must call.
+__device__ inline int last_index_not_after_warp(const int64_t *rowp, int R, int64_t bar, int64_t e0, int64_t eR) {
+    const int lane = threadIdx.x & 31;
+    constexpr int W = 32;
+    int ans = -2;                                                 // -2: not known yet
+    int lo = 1, hi = R - 1, a = 0;
+    if (!rowp) ans = -1;
+    else if (bar < e0) ans = -1;
+    else if (bar >= eR) ans = R - 1;
+    else {
+        int g = (int)((double)(bar - e0) * (double)(R - 1) / (double)(eR - e0));
+        g = max(0, min(g, R - 2));
+        a = max(0, min(g - W / 2 + 1, R - W)) & ~3;               // on a 32-byte boundary of the row
+    }
+    for (int it = 0; it < 3; ++it) {
+        const unsigned open = __ballot_sync(FULL, ans == -2);
+        if (!open) break;
+        // all the loads first, then the votes: the windows arrive together
+        int64_t v[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const unsigned long long pw = __shfl_sync(FULL, (unsigned long long)(uintptr_t)rowp, i);
+            const int ao = __shfl_sync(FULL, a, i);
+            const bool in = ((open >> i) & 1u) && ao + lane < R;
+            v[i] = in ? (int64_t)__ldg((const long long *)(uintptr_t)pw + ao + lane) : INT64_MAX;   // INT64_MAX: never <= bar (< 2^62)
+        }
+        int c = 0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const unsigned le = __ballot_sync(FULL, v[i] <= bar);
+            if (lane == i) c = __popc(le);
+        }
+        if (ans == -2) {
+            const int valid = min(W, R - a);
+            if (c > 0 && c < valid) ans = a + c - 1;              // the window holds the last element <= bar and its successor
+            else {
+                if (c == 0) hi = min(hi, a); else lo = max(lo, a + valid);
+                if (lo >= hi) ans = lo - 1;
+                else a = c == 0 ? max(0, hi - W) : min(lo, max(0, R - W));
+            }
+        }
+    }
+    if (ans == -2) {
+        // far off the guess: bisection between what the windows established (row[lo - 1] <= bar < row[hi])
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if ((int64_t)__ldg((const long long *)rowp + mid) <= bar) lo = mid + 1; else hi = mid;
+        }
+        ans = lo - 1;
+    }
+    return ans;
 }
 
 }  // namespace zl

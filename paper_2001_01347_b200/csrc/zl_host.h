@@ -15,7 +15,10 @@ inline int pow2_floor(int x) { int p = 1; while (p * 2 <= x) p *= 2; return p; }
 inline int pow2_ceil(int x) { int p = 1; while (p < x) p *= 2; return p; }
 
 // Shape of the segment sweep for one call.
-struct LaunchPlan { int threads, G, nseg, cap, target; size_t smem; };
+struct LaunchPlan {
+    int threads, G, nseg, cap, target; size_t smem;
+    int G_rest, target_rest;                                      // lanes per row and round size when a CTA of 512 threads runs the sweep
+};
 
 // Everything one call enqueues, for both the handle-based and the fixed-scratch entry points.
 struct Pipeline {
@@ -25,8 +28,9 @@ struct Pipeline {
     int filter_threads, filter_rows, filter_round;                // 0: automatic
     int pdl_off;                                                  // bit mask of kernels launched without early scheduling
     int prologue_threads, tail_threads;                           // 0: automatic
-    int fused;                                                    // RANGE filter route: one cluster launch instead of prologue, filter pass and tail
-    int cluster, filter_stages, prefetch_rows;                    // of the cluster kernel; 0: automatic
+    int cluster, filter_stages, filter_bulk;                      // 0: automatic (cluster: CTAs per instance of k_range_head; filter_bulk: 1 copy engine, 2 per-lane copies)
+    int tail_cap;                                                 // 0: default; else survivors the finishing CTA of the filter kernel has room for
+    int rest_per_sm;                                              // CTAs of k_range_rest resident per SM (0: ask the runtime)
     int checks_off;                                               // debug handle: unchecked kernels, clock stamps still taken
     int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;
 };
@@ -50,27 +54,38 @@ void launch_dep(bool early, void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
 // the filter and bucket stages fill in its per-call fields.  Each *_limits() raises the dynamic shared-memory
 // limit of its file's kernels (once per device).
 
-// prologue.cu: column scans (+ filter table), optional sortedness check
+// prologue.cu: column scans for the bucket route and the plain segment sweep; the optional sortedness check
 void enqueue_prologue(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const MatBatch &src);
 void enqueue_prologue(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const AriBatch &src);
+void enqueue_check_sorted(const Pipeline &q, cudaStream_t st);
 cudaError_t prologue_limits();
 
-// filter.cu: RANGE filter pass and the single-CTA finish of instances with few survivors; `mid` (may be null)
-// is recorded between the two
+// range_filter.cu: the RANGE filter route - k_range_head (summary, requests, filter table: a cluster per instance) and
+// k_range_filter (the filter pass in many small CTAs; the CTA that finishes an instance's last block also finishes an
+// instance with few survivors)
+cudaError_t enqueue_range_head(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const MatBatch &src);
+cudaError_t enqueue_range_head(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const AriBatch &src);
+cudaError_t enqueue_range_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const MatBatch &src);
+cudaError_t enqueue_range_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const AriBatch &src);
+cudaError_t enqueue_range_tail(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const MatBatch &src);
+cudaError_t enqueue_range_tail(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const AriBatch &src);
+int range_head_cluster_size(int B, int n, int num_sms, int gmax);
+cudaError_t range_limits();
+
+// filter.cu: the filter pass and the kernel that finishes instances with few survivors; `mid` is recorded between them
 void enqueue_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid, const MatBatch &src);
 void enqueue_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid, const AriBatch &src);
 cudaError_t filter_limits();
 
-// fused.cu: the RANGE filter route of an instance by one thread-block cluster in one launch (column scans, filter
-// table, filter pass, finish of instances with few survivors, index recovery)
-cudaError_t enqueue_fused(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const MatBatch &src);
-cudaError_t enqueue_fused(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const AriBatch &src);
-int fused_cluster_size(int B, int n, int num_sms, int gmax);
-cudaError_t fused_limits();
-
-// heavy.cu: RANGE instances with many survivors (cell scan, refinement, bucket sweep)
+// heavy.cu: the phases for RANGE instances with many survivors as kernels of their own (large shapes)
 void enqueue_heavy(const Pipeline &q, const FilterBufs &fb, cudaStream_t st);
 cudaError_t heavy_limits();
+
+// range_rest.cu: the route's last kernel - instances with many survivors (cell scan, refinement, bucket sweep), the segment
+// sweep of instances whose lists overflowed, and every instance's outputs
+cudaError_t enqueue_range_rest(const Pipeline &q, const FilterBufs &fb, const LaunchPlan &p, cudaStream_t st, const MatBatch &src);
+cudaError_t enqueue_range_rest(const Pipeline &q, const FilterBufs &fb, const LaunchPlan &p, cudaStream_t st, const AriBatch &src);
+cudaError_t range_rest_limits();
 
 // sum_route.cu: the bucket route (plan, index pass, bucket kernel); `mid` is recorded before the bucket kernel
 void enqueue_bucket_route(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid);

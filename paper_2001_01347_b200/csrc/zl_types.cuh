@@ -33,6 +33,15 @@ struct InstMeta {
     uint32_t dmin;       // no element whose own iteration (next - T) is this short can pass the filter table
 };
 
+// An instance's record read past the L1 cache: for kernels in which other CTAs update it between two of their phases.
+__device__ __forceinline__ InstMeta load_meta_cg(const InstMeta *p) {
+    static_assert(sizeof(InstMeta) == 64, "InstMeta is read as four 16-byte words");
+    union { InstMeta m; uint4 q[4]; } u;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) u.q[k] = __ldcg(reinterpret_cast<const uint4 *>(p) + k);
+    return u.m;
+}
+
 struct SegResult {
     uint64_t d;          // objective value of the segment's best candidate
     uint64_t t;          // its relative time (min(Z) for RANGE, the barrier for SUM)
@@ -88,11 +97,13 @@ struct FilterBufs {
     uint32_t *tilemax;   // [B][fcells/4096]  max of cellmax per tile of 4096 fine cells (scratch of the cell scan)
     uint32_t *rcnt;      // [B][nreg]         survivors per region (one region per CTA of the filter pass)
     uint64_t *list1;     // [B][list1cap]     survivors of the filter pass as (T << 32 | next), by region
-    uint32_t *flags;     // [3]               per call: some instance needs [0] scan/refine/buckets, [1] the segment sweep, [2] k_finalize
-    uint32_t *flags_next; // [3]              the flags of the handle's next call (the two sets alternate); zeroed by this call
-    uint64_t *part;      // [ctas][4]         fused kernel: per-CTA minima / maxima of the first and last column
-    uint32_t *ptab;      // [ctas][cells]     fused kernel: per-CTA partial filter tables
-    int32_t maxctas;     //                   CTAs the fused kernel's per-CTA records have room for
+    uint32_t *flags;     // [8]               per call: some instance needs [0] scan/refine/buckets, [1] the segment sweep; [4] arrivals at the
+                         //                   grid-wide barriers of the route's last kernel, [5] one of its barriers gave up
+    uint32_t *flags_next; // [8]              the flags of the handle's next call (the two sets alternate); zeroed by this call
+    uint64_t *part;      // [ctas][4]         k_range_head: per-CTA minima / maxima of the first and last column
+    uint32_t *done;      // [B]               blocks of the filter pass that have finished, per instance (in the end: how many it had)
+    uint32_t *ptab;      // [ctas][cells]     k_range_head: per-CTA partial filter tables
+    int32_t maxctas;     //                   CTAs k_range_head's per-CTA records have room for
     uint32_t *dbg;       // [4]               ZL_FLAG_DEBUG_CHECKS: record of the first index violation (0: none)
     uint32_t *bcnt;      // [B][nbk]          survivors of the refinement per bucket
     uint64_t *list2;     // [B][nbk][capb]    survivors of the refinement

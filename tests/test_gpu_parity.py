@@ -199,9 +199,7 @@ def test_host_detected_errors():
         h.set_option("no_such_option", 1)
     assert h.launches_per_call == 5 and h.workspace_bytes > 0      # tiny shape: prologue, plan, buckets, sweep, finalize
     h2 = zl.ZipLine(64, 128, 2)
-    assert h2.uses_cluster_kernel and h2.launches_per_call == 7     # the filter route: cluster kernel, heavy route (4), sweep, finalize
-    h2.set_option("no_fused", 1)
-    assert not h2.uses_cluster_kernel and h2.launches_per_call == 9 # prologue, filter, tail instead of the cluster kernel
+    assert h2.launches_per_call == 4                                 # the filter route: head, filter, tail, one last kernel
     h2.destroy()
     h.destroy()
 
