@@ -264,12 +264,12 @@ __global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBu
     const InstMeta M = meta[b];
     if (tid == 0) {
         // tell the later kernels of this call whether they have anything to do
-        const bool mine = M.status == ZL_OK && handled_by_filter(M, 1) && tail_instance(M);
+        const bool mine = M.status == ZL_OK && handled_by_filter(M, 1) && tail_instance(M, F);
         if (M.status == ZL_OK && !handled_by_filter(M, 1)) F.flags[1] = 1;
-        else if (M.status == ZL_OK && !tail_instance(M)) F.flags[0] = 1;
+        else if (M.status == ZL_OK && !tail_instance(M, F)) F.flags[0] = 1;
         if (!mine) F.flags[2] = 1;                                 // k_finalize has to write this instance's outputs
     }
-    if (M.status != ZL_OK || !handled_by_filter(M, 1) || !tail_instance(M)) return;
+    if (M.status != ZL_OK || !handled_by_filter(M, 1) || !tail_instance(M, F)) return;
     uint32_t *g = (uint32_t *)smem;                               // [cells]
     Key<uint32_t> *keys = (Key<uint32_t> *)(smem + (size_t)F.cells * 4);
     const BatchWS<uint32_t> ws{keys, keys + tcap, (uint32_t *)(keys + 2 * (size_t)tcap), tcap};
@@ -350,7 +350,10 @@ static void enqueue_filter_t(const Pipeline &q, FilterBufs &fb, cudaStream_t st,
     else
         launch_dep(!((q.pdl_off >> 1) & 1), k_filter, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.flags, (int)rpc, q.filter_round ? q.filter_round : 8, q.meta, fb);
     if (mid) cudaEventRecord(mid, st);
-    const int tcap = (int)std::min<long long>((long long)TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
+    // instances with at most tcap survivors are finished by one CTA each; with many instances a smaller limit lets more
+    // of those CTAs share an SM
+    const int tcap = (int)std::min<long long>(many ? (long long)TAIL_CAP / 2 : (long long)TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
+    fb.tailcap = tcap;
     launch_dep(!((q.pdl_off >> 2) & 1), k_tail<SRC>, dim3(q.B), dim3(q.tail_threads ? q.tail_threads : many ? (tcap <= 1024 ? 128 : 256) : std::max(64, std::min(1024, tcap / 2))), (size_t)tcap * 20 + (size_t)fb.cells * 4, st,
                (const InstMeta *)q.meta, fb, q.n, q.nres, q.seg, tcap, src, q.R, q.idx, q.barrier, q.wait, q.status);
 }

@@ -767,11 +767,11 @@ __global__ void __launch_bounds__(1024, 1) k_range_tail(const SRC src, const Ran
     const int n = P.n, R = P.R, cells = F.cells, tcap = P.tcap;
     const Guard<CHECK> gd{P.dbg, (uint32_t)b};
     const InstMeta M = P.meta[b];
-    const bool mine = M.status == ZL_OK && handled_by_filter(M, 1) && tail_instance(M);
+    const bool mine = M.status == ZL_OK && handled_by_filter(M, 1) && tail_instance(M, F);
     if (tid == 0) {
         // tell the last kernel of this call whether it has anything to do
         if (M.status == ZL_OK && !handled_by_filter(M, 1)) F.flags[1] = 1;
-        else if (M.status == ZL_OK && !tail_instance(M)) F.flags[0] = 1;
+        else if (M.status == ZL_OK && !tail_instance(M, F)) F.flags[0] = 1;
         if (!mine) F.flags[2] = 1;                                 // the last kernel has to write this instance's outputs
     }
     if (!mine) return;
@@ -944,11 +944,12 @@ static cudaError_t enqueue_range_filter_t(const Pipeline &q, FilterBufs &fb, cud
 }
 
 template <class SRC>
-static cudaError_t enqueue_range_tail_t(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const SRC &src) {
+static cudaError_t enqueue_range_tail_t(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const SRC &src) {
     RangeParams P;
     fill_params(P, q, fb);
-    P.tcap = (int)std::min<long long>((long long)TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
     const bool many = q.B > 2 * q.num_sms;
+    P.tcap = (int)std::min<long long>(many ? (long long)TAIL_CAP / 2 : (long long)TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
+    fb.tailcap = P.tcap;
     const int threads = q.tail_threads ? q.tail_threads : many ? (P.tcap <= 1024 ? 128 : 256) : std::max(64, std::min(1024, P.tcap / 2));
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
@@ -965,8 +966,8 @@ cudaError_t enqueue_range_head(const Pipeline &q, const FilterBufs &fb, cudaStre
 cudaError_t enqueue_range_head(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const AriBatch &src) { return enqueue_range_head_t(q, fb, st, src); }
 cudaError_t enqueue_range_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const MatBatch &src) { return enqueue_range_filter_t(q, fb, st, src); }
 cudaError_t enqueue_range_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const AriBatch &src) { return enqueue_range_filter_t(q, fb, st, src); }
-cudaError_t enqueue_range_tail(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const MatBatch &src) { return enqueue_range_tail_t(q, fb, st, src); }
-cudaError_t enqueue_range_tail(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const AriBatch &src) { return enqueue_range_tail_t(q, fb, st, src); }
+cudaError_t enqueue_range_tail(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const MatBatch &src) { return enqueue_range_tail_t(q, fb, st, src); }
+cudaError_t enqueue_range_tail(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const AriBatch &src) { return enqueue_range_tail_t(q, fb, st, src); }
 
 template <class SRC>
 static cudaError_t range_limits_t() {

@@ -19,7 +19,7 @@ static __device__ void heavy_tilemax(const InstMeta *meta, const FilterBufs &F, 
     for (int item = blockIdx.x; item < tiles * B; item += gridDim.x) {
         const int b = item / tiles, t = item % tiles;
         const InstMeta M = load_meta_cg(meta + b);
-        if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) continue;
+        if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M, F)) continue;
         const uint32_t *cmx = F.cellmax + (size_t)b * F.fcells + (size_t)t * SCAN_TILE;
         const int len = min(SCAN_TILE, F.fcells - t * SCAN_TILE);
         uint32_t loc = 0;
@@ -39,7 +39,7 @@ static __device__ void heavy_cellscan(const InstMeta *meta, const FilterBufs &F,
     for (int item = blockIdx.x; item < tiles * B; item += gridDim.x) {
         const int b = item / tiles, t = item % tiles;
         const InstMeta M = load_meta_cg(meta + b);
-        if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) continue;
+        if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M, F)) continue;
         uint32_t *cmx = F.cellmax + (size_t)b * F.fcells + (size_t)t * SCAN_TILE;
         const int len = min(SCAN_TILE, F.fcells - t * SCAN_TILE);
         uint32_t before = 0;
@@ -68,7 +68,7 @@ static __device__ void heavy_refine(InstMeta *meta, const FilterBufs &F, int B) 
     for (int item = blockIdx.x; item < F.nreg * B; item += gridDim.x) {
         const int b = item / F.nreg, reg = item % F.nreg;
         const InstMeta M = load_meta_cg(meta + b);
-        if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) continue;
+        if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M, F)) continue;
         const uint32_t m = F.rcnt[(size_t)b * F.nreg + reg];
         if (m == 0) continue;
         const uint32_t *g = F.cellmax + (size_t)b * F.fcells;     // G at fine cell starts
@@ -118,7 +118,7 @@ static __device__ void heavy_buckets(const InstMeta *meta, const FilterBufs &F, 
     const int b = item / ngroups, g = item % ngroups;
     __syncthreads();                                              // shared state of the previous item is done with
     const InstMeta M = load_meta_cg(meta + b);
-    if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M)) continue;
+    if (M.status != ZL_OK || !handled_by_filter(M, 1) || tail_instance(M, F)) continue;
     const uint32_t *bcnt = F.bcnt + (size_t)b * F.nbk;
     const uint32_t *g0 = F.cellmax + (size_t)b * F.fcells;        // G at fine cell starts (after heavy_cellscan)
     const uint64_t *list = F.list2 + (size_t)b * F.nbk * F.capb;

@@ -67,8 +67,8 @@ cudaError_t enqueue_range_head(const Pipeline &q, const FilterBufs &fb, cudaStre
 cudaError_t enqueue_range_head(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const AriBatch &src);
 cudaError_t enqueue_range_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const MatBatch &src);
 cudaError_t enqueue_range_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const AriBatch &src);
-cudaError_t enqueue_range_tail(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const MatBatch &src);
-cudaError_t enqueue_range_tail(const Pipeline &q, const FilterBufs &fb, cudaStream_t st, const AriBatch &src);
+cudaError_t enqueue_range_tail(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const MatBatch &src);
+cudaError_t enqueue_range_tail(const Pipeline &q, FilterBufs &fb, cudaStream_t st, const AriBatch &src);
 int range_head_cluster_size(int B, int n, int num_sms, int gmax);
 cudaError_t range_limits();
 

@@ -281,14 +281,14 @@ __device__ void finalize_rows(const SRC &src, int b, int rowchunk, int n, int R,
     const InstMeta M = f0.M;
     const uint64_t d0 = f0.d, t0 = f0.t;
     const unsigned long long vs0 = f0.vs;
-    if (filter == 1 && M.status == ZL_OK && handled_by_filter(M, 1) && tail_instance(M)) return;   // finished by the tail kernel
+    if (filter == 1 && M.status == ZL_OK && handled_by_filter(M, 1) && tail_instance(M, F)) return;   // finished by the tail kernel
     const RowEnds ends = pre ? *pre : row_ends(src, b, rowchunk, n, R);
     uint64_t bd = ~0ull, bt = ~0ull;
     uint32_t st = max((uint32_t)M.status, forced);
     if (st == ZL_OK) {
         const int used = !handled_by_filter(M, filter) ? nseg
                          : filter == 2 ? (int)M.count2 * F.ssub                         // bucket route: one result per part of a tile
-                         : tail_instance(M) ? 1 : (F.nbk + bucket_group(F, M.count2) - 1) / bucket_group(F, M.count2);
+                         : tail_instance(M, F) ? 1 : (F.nbk + bucket_group(F, M.count2) - 1) / bucket_group(F, M.count2);
         for (int s = lane; s < used; s += 32) {
             // past the L1 cache: another CTA of this kernel may have written it
             const unsigned long long *w = w0 + 3 * (size_t)s;

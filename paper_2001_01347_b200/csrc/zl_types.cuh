@@ -109,6 +109,7 @@ struct FilterBufs {
     uint64_t *list2;     // [B][nbk][capb]    survivors of the refinement
     int32_t cells, fcells, nbk, capb, grp;   // grp: fewest buckets per CTA of the bucket sweep
     int32_t nreg, regcap, list1cap;          // set per call: regions per instance and their capacity
+    int32_t tailcap;                         // set per call: most survivors of the filter pass the tail kernel finishes an instance with
     // SUM bucket route (all nullptr / 0 when the route is off): the timeline is cut into `scells` uniform
     // cells; runs of cells form buckets of about `sM` elements; `stiles` tiles of TILE_BK buckets each.
     uint32_t *bnd;                           // [B][stiles*15 + 1]   time at which each bucket starts (non-decreasing)
@@ -145,6 +146,6 @@ __device__ __forceinline__ uint32_t cell_of(uint32_t T, uint32_t cscale) { retur
 // Instances with at most this many survivors of the filter pass are finished by one CTA (k_tail);
 // larger ones go through cell scan, refinement and the bucket sweep.
 constexpr uint32_t TAIL_CAP = 2048;
-__device__ __forceinline__ bool tail_instance(const InstMeta &M) { return M.count <= TAIL_CAP; }
+__device__ __forceinline__ bool tail_instance(const InstMeta &M, const FilterBufs &F) { return M.count <= (uint32_t)F.tailcap; }
 
 }  // namespace zl
