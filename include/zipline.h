@@ -44,8 +44,10 @@ enum {
     ZL_FLAG_CHECK_SORTED = 1,  /* verify every row is non-decreasing (one extra pass over the input) */
     ZL_FLAG_FULL_SWEEP = 2,    /* examine every timestamp even where the search could stop early    */
     ZL_FLAG_PREDICTOR = 4,     /* the handle also holds a [max_batch][n][R] buffer for zl_predict_select_batched */
-    ZL_FLAG_DEBUG_CHECKS = 8   /* kernels test every computed index against its buffer before using it and record the
+    ZL_FLAG_DEBUG_CHECKS = 8,  /* kernels test every computed index against its buffer before using it and record the
                                   first violation instead of making the access (see zl_debug_report in zipline_debug.h) */
+    ZL_FLAG_FORCE_FILTER = 16  /* RANGE: take the filter route even for instances small enough to be sorted whole
+                                  (for tests: the route's kernels on shapes a brute-force search can check)        */
 };
 
 typedef struct {
@@ -62,7 +64,13 @@ typedef struct {
  * n x R timestamps (Section IV: the n x R matrix M, one row per worker).
  * cfg and out are host pointers.  ZL_ERR_UNSUPPORTED if n exceeds
  * zl_max_workers().  The handle is not thread safe; distinct handles are
- * independent.
+ * independent.  The caller's current device is the same after the call as before it.
+ *
+ * Ordering: a handle has ONE set of scratch buffers, and every call on it reads and
+ * writes them on the device.  Two calls on the same handle must therefore run one
+ * after the other on the device: issue them on one stream, or order them with events.
+ * Calls on one handle from two streams (or two host threads) without such ordering race
+ * on the scratch and give wrong results; nothing detects it.  Use a handle per stream.
  */
 zl_status zl_create(const zl_config *cfg, zl_handle **out);
 
@@ -85,7 +93,8 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out);
  *             instance in error gets idx = -1 and barrier = wait = INT64_MIN.
  *   cuda_stream  a cudaStream_t (0 = default stream).  The call only enqueues work
  *             and returns; outputs are valid once the stream has run.  It never
- *             allocates or synchronises.  The caller owns every buffer.
+ *             allocates or synchronises.  The caller owns every buffer.  The current
+ *             device must be the handle's (cfg.device): ZL_ERR_INVALID_ARG otherwise.
  *
  * Result definition: wait is the minimum of d_Z over all R^n selections;
  * barrier is the smallest max(Z) among the minimisers; idx[p] is the largest i

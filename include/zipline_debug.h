@@ -54,6 +54,15 @@ zl_status zl_probe_read_batched(const int64_t *d_ts, const int32_t *d_count, int
 zl_status zl_filter_counts(zl_handle *h, int32_t B, uint32_t *h_filtered, uint32_t *h_refined, uint32_t *h_overflow);
 
 /*
+ * A handle created with ZL_FLAG_DEBUG_CHECKS puts 64 bytes of a fixed pattern behind every scratch buffer it
+ * allocates.  No kernel may write there: a changed byte means that some store ran past the end of its buffer
+ * without an index check seeing it.  Waits for the device, reads the patterns back and reports how many buffers
+ * carry one (*buffers; 0 for a handle without the flag) and how many of them are damaged (*damaged).  Host
+ * pointers.  The patterns are not repaired.
+ */
+zl_status zl_check_canaries(zl_handle *h, int32_t *buffers, int32_t *damaged);
+
+/*
  * Self-checks (no counterpart in the paper; the stand-in for a memory checker).  A handle created with
  * ZL_FLAG_DEBUG_CHECKS runs kernels in which every computed index into global or shared memory, and every bulk
  * copy, is compared with the extent of its buffer first; an index out of range is not used (the access is

@@ -16,7 +16,7 @@ from . import build as _build
 ZL_OK = 0
 ZL_ERR_INVALID_ARG, ZL_ERR_UNSUPPORTED, ZL_ERR_NOMEM, ZL_ERR_CUDA, ZL_ERR_UNSORTED, ZL_ERR_TIMEOUT = range(1, 7)
 ZL_OBJ_RANGE, ZL_OBJ_SUM = 0, 1
-ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP, ZL_FLAG_PREDICTOR, ZL_FLAG_DEBUG_CHECKS = 1, 2, 4, 8
+ZL_FLAG_CHECK_SORTED, ZL_FLAG_FULL_SWEEP, ZL_FLAG_PREDICTOR, ZL_FLAG_DEBUG_CHECKS, ZL_FLAG_FORCE_FILTER = 1, 2, 4, 8, 16
 
 EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace_batched", "zl_destroy",
            "zl_set_option", "zl_status_string", "zl_workspace_bytes", "zl_launches_per_call",
@@ -24,7 +24,7 @@ EXPORTS = ("zl_create", "zl_select_batched", "zl_select_batched_host", "zl_trace
            "zl_profile_begin", "zl_profile_read", "zl_profile_end",
            "zl_select_batched_noalloc", "zl_noalloc_max_batch", "zl_noalloc_scratch_bytes", "zl_filter_counts",
            "zl_predict_batched", "zl_predict_select_batched", "zl_gridscan_batched", "zl_route",
-           "zl_probe_read_batched", "zl_debug_report", "zl_debug_stamps")
+           "zl_probe_read_batched", "zl_debug_report", "zl_debug_stamps", "zl_check_canaries")
 
 
 class zl_config(ctypes.Structure):
@@ -63,6 +63,8 @@ def _load() -> ctypes.CDLL:
     lib.zl_predict_select_batched.restype = ctypes.c_int
     lib.zl_filter_counts.argtypes = [vp, i32, vp, vp, vp]
     lib.zl_filter_counts.restype = ctypes.c_int
+    lib.zl_check_canaries.argtypes = [vp, vp, vp]
+    lib.zl_check_canaries.restype = ctypes.c_int
     lib.zl_debug_report.argtypes = [vp, vp]
     lib.zl_debug_report.restype = ctypes.c_int
     lib.zl_debug_stamps.argtypes = [vp, i32, vp]
@@ -210,6 +212,13 @@ class ZipLine:
                "zl_filter_counts")
         return list(f), list(r), list(o)
 
+    def check_canaries(self):
+        """(buffers, damaged): scratch buffers of a ZL_FLAG_DEBUG_CHECKS handle that end in canary bytes, and how
+        many of those have been written over.  Synchronises."""
+        nb, bad = ctypes.c_int32(0), ctypes.c_int32(0)
+        _check(lib.zl_check_canaries(self._h, ctypes.addressof(nb), ctypes.addressof(bad)), "zl_check_canaries")
+        return int(nb.value), int(bad.value)
+
     def debug_report(self):
         """(code, cta, index) of the first index violation since the last report, (0, 0, 0) if none.  Synchronises."""
         rec = (ctypes.c_uint32 * 4)()
@@ -217,7 +226,7 @@ class ZipLine:
         return int(rec[0]), int(rec[1]), int(rec[2]) | (int(rec[3]) << 32)
 
     def debug_stamps(self, ctas: int):
-        """[ctas, 16] uint64 nanosecond stamps of the cluster kernel's phase boundaries in the last call (numpy)."""
+        """[ctas, 16] uint64 nanosecond stamps of the RANGE filter route's phase boundaries in the last call (numpy)."""
         import numpy as np
         out = np.zeros((ctas, 16), dtype=np.uint64)
         _check(lib.zl_debug_stamps(self._h, ctas, out.ctypes.data), "zl_debug_stamps")

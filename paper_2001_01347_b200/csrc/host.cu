@@ -43,13 +43,16 @@ struct zl_handle {
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round, opt_cluster, opt_filter_stages, opt_checks_off, opt_filter_bulk, opt_tail_cap;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round, opt_cluster, opt_filter_stages, opt_checks_off, opt_filter_bulk, opt_tail_cap, opt_max_rounds;
     int epoch;               // calls so far: the two sets of per-call flags alternate
     int last_cuda_error;
     int launches;
     // optional per-kernel timing: PROF_EVENTS events per recorded call
     cudaEvent_t *prof_ev;
     int prof_cap, prof_calls;
+    // ZL_FLAG_DEBUG_CHECKS: every scratch buffer ends in CANARY_BYTES bytes of a fixed pattern that no kernel may touch
+    unsigned char *canary[24];
+    int ncanary;
 };
 
 namespace {
@@ -59,6 +62,8 @@ using zl::Pipeline;
 using zl::pow2_ceil;
 using zl::pow2_floor;
 constexpr int PROF_EVENTS = 5;
+constexpr size_t CANARY_BYTES = 64;
+constexpr int CANARY_BYTE = 0xC5;
 
 // SRC: zl::MatBatch (the rows are read from q.ts) or zl::AriBatch (predicted rows, generated on the fly; RANGE, filter
 // route or plain segment sweep only).
@@ -161,6 +166,23 @@ zl_status cuda_fail(zl_handle *h, cudaError_t e) {
     return e == cudaErrorMemoryAllocation ? ZL_ERR_NOMEM : ZL_ERR_CUDA;
 }
 
+// Makes `device` current for the life of the object and puts the caller's device back afterwards.
+struct DeviceScope {
+    int prev = -1;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceScope(int device) {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != device) err = cudaSetDevice(device); else if (err == cudaSuccess) prev = -1;
+    }
+    ~DeviceScope() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// The stream-ordered entry points only enqueue work: the caller's current device must be the handle's.
+bool on_device(int device) {
+    int cur = -1;
+    return cudaGetDevice(&cur) == cudaSuccess && cur == device;
+}
+
 #define ZL_CUDA(h, call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail((h), e_); } while (0)
 
 }  // namespace
@@ -187,7 +209,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     *out = nullptr;
     if (cfg->n_workers < 1 || cfg->lookahead_R < 1 || cfg->max_batch < 1) return ZL_ERR_INVALID_ARG;
     if (cfg->objective != ZL_OBJ_RANGE && cfg->objective != ZL_OBJ_SUM) return ZL_ERR_INVALID_ARG;
-    if (cfg->flags & ~(ZL_FLAG_CHECK_SORTED | ZL_FLAG_FULL_SWEEP | ZL_FLAG_PREDICTOR | ZL_FLAG_DEBUG_CHECKS)) return ZL_ERR_INVALID_ARG;
+    if (cfg->flags & ~(ZL_FLAG_CHECK_SORTED | ZL_FLAG_FULL_SWEEP | ZL_FLAG_PREDICTOR | ZL_FLAG_DEBUG_CHECKS | ZL_FLAG_FORCE_FILTER)) return ZL_ERR_INVALID_ARG;
     if (cfg->n_workers > zl::MAX_WORKERS) return ZL_ERR_UNSUPPORTED;
     if ((long long)cfg->n_workers * cfg->lookahead_R > (1LL << 31) - 1) return ZL_ERR_UNSUPPORTED;
     if (cfg->max_batch > 65535) return ZL_ERR_UNSUPPORTED;
@@ -197,13 +219,25 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     if (!h) return ZL_ERR_NOMEM;
     memset(h, 0, sizeof(*h));
     h->cfg = *cfg;
-    cudaError_t e = cudaSetDevice(cfg->device);
+    DeviceScope scope(cfg->device);                               // the caller's device is current again on return
+    cudaError_t e = scope.err;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&h->num_sms, cudaDevAttrMultiProcessorCount, cfg->device);
+    // scratch buffers; a debug handle's end in canary bytes (zl_check_canaries)
+    const bool canaries = (cfg->flags & ZL_FLAG_DEBUG_CHECKS) != 0;
+    auto alloc = [&](void **ptr, size_t bytes) -> cudaError_t {
+        if (!canaries) return cudaMalloc(ptr, bytes);
+        const size_t body = (bytes + 15) & ~(size_t)15;
+        cudaError_t a = cudaMalloc(ptr, body + CANARY_BYTES);
+        if (a == cudaSuccess) a = cudaMemset((unsigned char *)*ptr + body, CANARY_BYTE, CANARY_BYTES);
+        if (a == cudaSuccess && h->ncanary < 24) h->canary[h->ncanary++] = (unsigned char *)*ptr + body;
+        return a;
+    };
     const size_t meta_b = (size_t)cfg->max_batch * sizeof(zl::InstMeta);
     size_t filter_b = 0;
     h->nres = zl::MAX_SEGMENTS;
     // RANGE instances that fit one shared-memory batch are sorted whole by the bucket route; larger ones take the filter route
-    const bool range_small = cfg->objective == ZL_OBJ_RANGE && (long long)cfg->n_workers * cfg->lookahead_R <= 4096;
+    const bool range_small = cfg->objective == ZL_OBJ_RANGE && (long long)cfg->n_workers * cfg->lookahead_R <= 4096 &&
+                             !(cfg->flags & ZL_FLAG_FORCE_FILTER);
     if (cfg->objective == ZL_OBJ_RANGE && !range_small) {
         const long long N = (long long)cfg->n_workers * cfg->lookahead_R;
         const size_t mb = (size_t)cfg->max_batch;
@@ -229,14 +263,14 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
                            (void **)&f.part, (void **)&f.ptab, (void **)&f.done};
         f.maxctas = (int)std::min<size_t>(ctas, 0x7fffffff);
         for (int i = 0; i < 12; ++i) {
-            if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
+            if (e == cudaSuccess) e = alloc(ptrs[i], sizes[i]);
             filter_b += sizes[i];
         }
         if (e == cudaSuccess) e = cudaMemset(f.flags, 0, 64);
         if (cfg->flags & ZL_FLAG_DEBUG_CHECKS) {
             // the violation record, then 16 clock stamps per CTA of the head kernel and of the filter kernel
             const size_t dbg_b = 64 + (ctas + mb * ((size_t)cfg->n_workers + 1) / 2 + 1) * 16 * 8;
-            if (e == cudaSuccess) e = cudaMalloc((void **)&f.dbg, dbg_b);
+            if (e == cudaSuccess) e = alloc((void **)&f.dbg, dbg_b);
             if (e == cudaSuccess) e = cudaMemset(f.dbg, 0, dbg_b);
             filter_b += dbg_b;
         }
@@ -261,7 +295,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
             const size_t sizes[4] = {mb * nb1 * 4, 64, f.scells ? mb * f.stiles * cfg->n_workers * 32 : 64, 64};
             void **ptrs[4] = {(void **)&f.bnd, (void **)&f.cellacc, (void **)&f.itab, (void **)&f.flags};
             for (int i = 0; i < 4; ++i) {
-                if (e == cudaSuccess) e = cudaMalloc(ptrs[i], sizes[i]);
+                if (e == cudaSuccess) e = alloc(ptrs[i], sizes[i]);
                 filter_b += sizes[i];
             }
             if (e == cudaSuccess) e = cudaMemset(f.flags, 0, 64);
@@ -271,10 +305,10 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         }
     }
     const size_t seg_b = (size_t)cfg->max_batch * h->nres * sizeof(zl::SegResult);
-    if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_meta, meta_b);
-    if (e == cudaSuccess) e = cudaMalloc((void **)&h->d_seg, seg_b);
+    if (e == cudaSuccess) e = alloc((void **)&h->d_meta, meta_b);
+    if (e == cudaSuccess) e = alloc((void **)&h->d_seg, seg_b);
     const size_t pred_b = (cfg->flags & ZL_FLAG_PREDICTOR) ? (size_t)cfg->max_batch * cfg->n_workers * cfg->lookahead_R * 8 : 0;
-    if (e == cudaSuccess && pred_b) e = cudaMalloc((void **)&h->d_pred, pred_b);
+    if (e == cudaSuccess && pred_b) e = alloc((void **)&h->d_pred, pred_b);
     if (e == cudaSuccess) e = raise_shared_memory_limits();   // more than the default 48 KB of dynamic shared memory
     if (e != cudaSuccess) {
         zl_status st = cuda_fail(nullptr, e);
@@ -304,7 +338,8 @@ zl_status zl_profile_end(zl_handle *h) {
 zl_status zl_profile_begin(zl_handle *h, int32_t max_calls) {
     if (!h || max_calls < 1 || max_calls > 65536) return ZL_ERR_INVALID_ARG;
     zl_profile_end(h);
-    ZL_CUDA(h, cudaSetDevice(h->cfg.device));
+    DeviceScope scope(h->cfg.device);
+    ZL_CUDA(h, scope.err);
     h->prof_ev = new (std::nothrow) cudaEvent_t[PROF_EVENTS * (size_t)max_calls];
     if (!h->prof_ev) return ZL_ERR_NOMEM;
     for (int i = 0; i < PROF_EVENTS * max_calls; ++i) {
@@ -323,6 +358,8 @@ zl_status zl_profile_begin(zl_handle *h, int32_t max_calls) {
 
 zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_stage) {
     if (!h || !calls || !ms_stage) return ZL_ERR_INVALID_ARG;
+    DeviceScope scope(h->cfg.device);
+    ZL_CUDA(h, scope.err);
     *calls = h->prof_calls;
     for (int k = 0; k < PROF_EVENTS - 1; ++k) ms_stage[k] = 0.f;
     for (int c = 0; c < h->prof_calls; ++c) {
@@ -340,7 +377,7 @@ zl_status zl_profile_read(zl_handle *h, int32_t *calls, float *ms_stage) {
 
 zl_status zl_destroy(zl_handle *h) {
     if (!h) return ZL_OK;
-    cudaSetDevice(h->cfg.device);
+    DeviceScope scope(h->cfg.device);
     cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
     cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
     cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
@@ -375,6 +412,8 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
     } else if (!strcmp(key, "filter_bulk")) {
         if (value > 2) return ZL_ERR_INVALID_ARG;
         h->opt_filter_bulk = value;
+    } else if (!strcmp(key, "max_rounds")) {
+        h->opt_max_rounds = value;                  // the segment sweep gives up (ZL_ERR_TIMEOUT) after this many rounds of a segment
     } else if (!strcmp(key, "tail_cap")) {
         if (value != 0 && (value < 64 || value > 2048 || (value & (value - 1)))) return ZL_ERR_INVALID_ARG;
         h->opt_tail_cap = (int)value;
@@ -425,6 +464,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     if (((uintptr_t)d_ts & 7) || ((uintptr_t)d_barrier & 7) || ((uintptr_t)d_wait & 7) || ((uintptr_t)d_idx & 3) ||
         ((uintptr_t)d_status & 3))
         return ZL_ERR_INVALID_ARG;
+    if (!on_device(h->cfg.device)) return ZL_ERR_INVALID_ARG;     // the launches would go to another GPU than the handle's buffers
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const int n = h->cfg.n_workers, R = h->cfg.lookahead_R, obj = h->cfg.objective;
     const LaunchPlan p = make_plan(h, B);
@@ -439,7 +479,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
     if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
     q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
-    q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0;
+    q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds;
     if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
         uint32_t *base = h->fb.flags;
         q.fb.flags = base + 8 * (h->epoch & 1);
@@ -457,9 +497,28 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
 zl_status zl_debug_stamps(zl_handle *h, int32_t ctas, uint64_t *h_stamps) {
     if (!h || !h_stamps || ctas < 1) return ZL_ERR_INVALID_ARG;
     if (!h->fb.dbg || ctas > (long long)h->fb.maxctas + ((long long)h->cfg.max_batch * (h->cfg.n_workers + 1)) / 2) return ZL_ERR_INVALID_ARG;
-    ZL_CUDA(h, cudaSetDevice(h->cfg.device));
+    DeviceScope scope(h->cfg.device);
+    ZL_CUDA(h, scope.err);
     ZL_CUDA(h, cudaDeviceSynchronize());
     ZL_CUDA(h, cudaMemcpy(h_stamps, h->fb.dbg + 16, (size_t)ctas * 16 * 8, cudaMemcpyDeviceToHost));
+    return ZL_OK;
+}
+
+zl_status zl_check_canaries(zl_handle *h, int32_t *buffers, int32_t *damaged) {
+    if (!h || !buffers || !damaged) return ZL_ERR_INVALID_ARG;
+    *buffers = h->ncanary;
+    *damaged = 0;
+    if (!h->ncanary) return ZL_OK;
+    DeviceScope scope(h->cfg.device);
+    ZL_CUDA(h, scope.err);
+    ZL_CUDA(h, cudaDeviceSynchronize());
+    for (int i = 0; i < h->ncanary; ++i) {
+        unsigned char tail[CANARY_BYTES];
+        ZL_CUDA(h, cudaMemcpy(tail, h->canary[i], CANARY_BYTES, cudaMemcpyDeviceToHost));
+        bool ok = true;
+        for (size_t k = 0; k < CANARY_BYTES; ++k) ok = ok && tail[k] == (unsigned char)CANARY_BYTE;
+        if (!ok) ++*damaged;
+    }
     return ZL_OK;
 }
 
@@ -467,7 +526,8 @@ zl_status zl_debug_report(zl_handle *h, uint32_t *h_record) {
     if (!h || !h_record) return ZL_ERR_INVALID_ARG;
     memset(h_record, 0, 4 * sizeof(uint32_t));
     if (!h->fb.dbg) return ZL_OK;
-    ZL_CUDA(h, cudaSetDevice(h->cfg.device));
+    DeviceScope scope(h->cfg.device);
+    ZL_CUDA(h, scope.err);
     ZL_CUDA(h, cudaDeviceSynchronize());
     ZL_CUDA(h, cudaMemcpy(h_record, h->fb.dbg, 4 * sizeof(uint32_t), cudaMemcpyDeviceToHost));
     ZL_CUDA(h, cudaMemset(h->fb.dbg, 0, 4 * sizeof(uint32_t)));
@@ -476,7 +536,8 @@ zl_status zl_debug_report(zl_handle *h, uint32_t *h_record) {
 
 zl_status zl_filter_counts(zl_handle *h, int32_t B, uint32_t *h_filtered, uint32_t *h_refined, uint32_t *h_overflow) {
     if (!h || B < 1 || B > h->cfg.max_batch) return ZL_ERR_INVALID_ARG;
-    ZL_CUDA(h, cudaSetDevice(h->cfg.device));
+    DeviceScope scope(h->cfg.device);
+    ZL_CUDA(h, scope.err);
     ZL_CUDA(h, cudaDeviceSynchronize());
     uint32_t *dst[3] = {h_filtered, h_refined, h_overflow};
     const size_t off[3] = {offsetof(zl::InstMeta, count), offsetof(zl::InstMeta, count2), offsetof(zl::InstMeta, overflow)};
@@ -492,6 +553,7 @@ zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const i
                                     void *cuda_stream) {
     if (!h || !h->d_pred) return ZL_ERR_INVALID_ARG;
     if (B < 1 || B > h->cfg.max_batch) return ZL_ERR_INVALID_ARG;
+    if (!on_device(h->cfg.device)) return ZL_ERR_INVALID_ARG;
     if (h->cfg.objective == ZL_OBJ_RANGE && h->fb.table != nullptr) {
         // the filter route (and its fallback) on generated rows: the predicted matrix is never written
         if (!d_last || !d_interval || !d_idx || !d_barrier || !d_wait) return ZL_ERR_INVALID_ARG;
@@ -510,7 +572,7 @@ zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const i
         q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
         if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
         q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
-        q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0;
+        q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds;
         if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
             uint32_t *base = h->fb.flags;
             q.fb.flags = base + 8 * (h->epoch & 1);
@@ -535,7 +597,8 @@ zl_status zl_select_batched_host(zl_handle *h, const int64_t *h_ts, int32_t B, i
     if (!h || !h_ts || !h_idx || !h_barrier || !h_wait) return ZL_ERR_INVALID_ARG;
     if (B < 1 || B > h->cfg.max_batch) return ZL_ERR_INVALID_ARG;
     const size_t n = h->cfg.n_workers, R = h->cfg.lookahead_R, mb = h->cfg.max_batch;
-    ZL_CUDA(h, cudaSetDevice(h->cfg.device));
+    DeviceScope scope(h->cfg.device);
+    ZL_CUDA(h, scope.err);
     if (!h->s_ts) {
         ZL_CUDA(h, cudaStreamCreateWithFlags(&h->s_stream, cudaStreamNonBlocking));
         ZL_CUDA(h, cudaMalloc((void **)&h->s_ts, mb * n * R * 8));
@@ -635,7 +698,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
     q.meta = meta; q.seg = seg; q.nres = p.nseg;
     memset(&q.fb, 0, sizeof(q.fb));
-    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0; q.cluster = q.filter_stages = 0; q.checks_off = 0; q.filter_bulk = 0; q.tail_cap = 0; q.rest_per_sm = 0;
+    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0; q.cluster = q.filter_stages = 0; q.checks_off = 0; q.filter_bulk = 0; q.tail_cap = 0; q.rest_per_sm = 0; q.max_rounds = 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr, zl::MatBatch{d_ts});
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;

@@ -95,6 +95,7 @@ static cudaError_t enqueue_range_rest_t(const Pipeline &q, const FilterBufs &fb,
     sp.n = q.n; sp.R = q.R; sp.B = q.B; sp.nseg = p.nseg; sp.nres = q.nres; sp.G = p.G_rest; sp.cap = p.cap;
     sp.flags = q.flags; sp.target = p.target_rest; sp.filter = 1;
     sp.need = nullptr;
+    sp.max_rounds = q.max_rounds;
     RestParams P;
     P.n = q.n; P.R = q.R; P.B = q.B; P.nres = q.nres; P.nseg = p.nseg;
     P.idx = q.idx; P.barrier = q.barrier; P.wait = q.wait; P.status = q.status;

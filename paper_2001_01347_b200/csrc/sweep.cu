@@ -33,6 +33,7 @@ static void enqueue_sweep_t(const Pipeline &q, const FilterBufs &fb, const Launc
     sp.n = q.n; sp.R = q.R; sp.B = q.B; sp.nseg = p.nseg; sp.nres = q.nres; sp.G = p.G; sp.cap = p.cap;
     sp.flags = q.flags; sp.target = p.target; sp.filter = fast ? 1 : 0;
     sp.need = fast ? fb.flags : nullptr;
+    sp.max_rounds = q.max_rounds;
     // with a fast route on, the segment sweep is only the fallback: a small persistent grid
     const int items = p.nseg * q.B;
     const int sweep_ctas = fast ? std::min(items, 2 * q.num_sms) : items;

@@ -30,6 +30,7 @@ struct Pipeline {
     int prologue_threads, tail_threads;                           // 0: automatic
     int cluster, filter_stages, filter_bulk;                      // 0: automatic (cluster: CTAs per instance of k_range_head; filter_bulk: 1 copy engine, 2 per-lane copies)
     int tail_cap;                                                 // 0: default; else survivors the finishing CTA of the filter kernel has room for
+    int max_rounds;                                               // 0: automatic; else the segment sweep's round limit
     int rest_per_sm;                                              // CTAs of k_range_rest resident per SM (0: ask the runtime)
     int checks_off;                                               // debug handle: unchecked kernels, clock stamps still taken
     int32_t *idx; int64_t *barrier; int64_t *wait; int32_t *status;

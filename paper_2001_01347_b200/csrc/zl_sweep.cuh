@@ -94,12 +94,17 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const ROW
         // nominal round: `target` elements out of the segment's share of the instance
         uint64_t delta = max((uint64_t)1, (seg_hi - seg_lo) / max((uint64_t)1, ((uint64_t)n * R / P.nseg) / max(1, P.target)));
         uint32_t count_before = 0;
+        // Every round either commits (and then consumes an element, or moves the window to the next one: at most
+        // n * R + 1 of those a segment) or does not fit: then it flushes the batch, or halves the window, which is at
+        // least 1 and fits once it holds one element a row (the batch has room for that), so fewer than 70 rounds in
+        // a row can fail to commit.  A segment that goes past either bound reports ZL_ERR_TIMEOUT instead of looping.
         uint64_t rounds = 0;
-        const uint64_t max_rounds = 4 * (uint64_t)n * R + 4096;
+        uint32_t stalled = 0;
+        const uint64_t max_rounds = P.max_rounds > 0 ? (uint64_t)P.max_rounds : 72 * ((uint64_t)n * R + 2);
 
         while (rlo < seg_hi) {
             if (OBJ == ZL_OBJ_RANGE && cut && floorv == INF) break;     // a row ran out: no later Z is complete
-            if (++rounds > max_rounds) { status = ZL_ERR_TIMEOUT; break; }
+            if (++rounds > max_rounds || stalled > 72) { status = ZL_ERR_TIMEOUT; break; }
             const uint64_t rhi64 = min(rlo + delta, seg_hi);
             const K rhi = (K)rhi64;
             if (tid == 0) { sh.overflow = 0; sh.consumed = 0; sh.minhead = ~0ull; }
@@ -171,6 +176,7 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const ROW
             const K vmax = (K)sh.vmax;
             __syncthreads();
             if (overflow) {
+                ++stalled;
                 // the round does not fit: flush what was there, or shorten the window; cursors are not committed
                 if (count_before > 0) {
                     run_batch<K, OBJ>(ws, (int)count_before, t0, n, sh.tmp, carryMax, carryS, carryC, bd, bt);
@@ -184,6 +190,7 @@ __device__ void sweep_segment(const SweepParams &P, const InstMeta &M, const ROW
                 continue;
             }
             // commit the round
+            stalled = 0;
             { uint32_t *t = cur; cur = nxt; nxt = t; }
             count_before = count;
             if (OBJ == ZL_OBJ_RANGE) floorv = max(floorv, vmax);

@@ -126,6 +126,7 @@ struct SweepParams {
     int32_t n, R, B, nseg, nres, G, cap, flags, target;   // nres: SegResult slots per instance
     int32_t filter;      // instances handled by the filter route are skipped
     const uint32_t *need; // filter on: [1] != 0 when some instance needs this sweep; nullptr: always run
+    int32_t max_rounds;   // 0: the bound that follows from the input's size; else rounds a segment may take before ZL_ERR_TIMEOUT
 };
 
 // Buckets per CTA of the bucket sweep for an instance with `count` refined survivors: the static

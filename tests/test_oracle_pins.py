@@ -249,6 +249,25 @@ def test_trace_matches_the_selection():
         for q in range(k + 1):
             last[int(tr["om_p"][q])] = int(tr["om_t"][q])
         assert tr["S"][k] == sum(last.values()) and tr["cnt"][k] == len(last)
+        # every array at every position, straight from its definition (no running state)
+        N = n * R
+        INF, NINF = np.iinfo(np.int64).max, np.iinfo(np.int64).min
+        t0 = int(M[:, 0].max())
+        for q in range(N):
+            wp, wi, wt = int(tr["om_p"][q]), int(tr["om_i"][q]), int(tr["om_t"][q])
+            assert tr["delta"][q] == (wt if wi == 0 else wt - int(M[wp, wi - 1]))
+            assert tr["first"][q] == (1 if wi == 0 else 0)
+            assert tr["next"][q] == (INF if wi == R - 1 else int(M[wp, wi + 1]))
+            before = [INF if int(tr["om_i"][j]) == R - 1 else int(M[int(tr["om_p"][j]), int(tr["om_i"][j]) + 1]) for j in range(q)]
+            pm = max(before) if before else NINF
+            assert tr["PM"][q] == pm
+            latest = {}
+            for j in range(q + 1):
+                latest[int(tr["om_p"][j])] = int(tr["om_t"][j])
+            assert tr["S"][q] == sum(latest.values()) and tr["cnt"][q] == len(latest)
+            g = max(wt, t0, pm)
+            assert tr["d_range"][q] == (INF if g == INF else g - wt)
+            assert tr["w_sum"][q] == (n * wt - sum(latest.values()) if len(latest) == n else INF)
         # minimum over positions reproduces the selection, with the first-minimum rule
         w, b, _ = o.sweep(M, o.RANGE)
         d = tr["d_range"]

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle as o
 import zl_inputs as zi
 
 pytestmark = pytest.mark.gpu
@@ -44,6 +45,30 @@ def test_noalloc_matches_handle_path_on_two_calls_in_a_row(objective):
         assert torch.equal(got.barrier, ref.barrier)
         assert torch.equal(got.wait, ref.wait)
         h.destroy()
+
+
+@pytest.mark.parametrize("objective", [0, 1])
+def test_noalloc_against_the_oracle_with_a_bad_instance_and_the_sortedness_check(objective):
+    w = zi.CONFIGS["c2"].with_(B=5, n=12, R=40)
+    ts = zi.generate(w)
+    ts[3, 7, 0] = -9                      # a negative timestamp: this instance alone is refused
+    got = zl.zl_select_batched_noalloc(torch.from_numpy(ts).cuda(), _empty_selection(w.B, w.n), objective)
+    torch.cuda.synchronize()
+    status = got.status.cpu().numpy()
+    assert status.tolist() == [0, 0, 0, zl.binding.ZL_ERR_INVALID_ARG, 0]
+    assert (got.idx.cpu().numpy()[3] == -1).all()
+    for b in (0, 1, 2, 4):
+        wt, bar, ix = o.sweep(ts[b], objective)
+        assert (int(got.wait[b]), int(got.barrier[b])) == (wt, bar) and (got.idx[b].cpu().numpy() == ix).all()
+    # with the sortedness check: a row that goes backwards is reported for its instance only
+    ts2 = zi.generate(w)
+    ts2[1, 2, 5] = ts2[1, 2, 3] - 1
+    got = zl.zl_select_batched_noalloc(torch.from_numpy(ts2).cuda(), _empty_selection(w.B, w.n), objective, zl.ZL_FLAG_CHECK_SORTED)
+    torch.cuda.synchronize()
+    assert got.status.cpu().tolist() == [0, zl.binding.ZL_ERR_UNSORTED, 0, 0, 0]
+    for b in (0, 2, 3, 4):
+        wt, bar, ix = o.sweep(ts2[b], objective)
+        assert (int(got.wait[b]), int(got.barrier[b])) == (wt, bar) and (got.idx[b].cpu().numpy() == ix).all()
 
 
 def test_noalloc_rejects_batches_beyond_the_fixed_scratch():
