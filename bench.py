@@ -177,9 +177,10 @@ def run_reference(args, w, objective):
 
 
 STAGES = {  # names of what runs between the library's stage events, by route
-    1: ("k_range_head", "k_range_filter", "k_tilemax+k_cellscan+k_refine+k_buckets+k_sweep", "k_finalize"),
+    1: ("k_range_head", "k_filter", "k_tail", "k_range_rest"),     # large shapes: the last stage is one kernel per phase
     2: ("k_prologue", "k_sum_plan+k_sum_index", "k_sum_buckets+k_sweep", "k_finalize"),
     0: ("k_prologue", "-", "k_sweep", "k_finalize"),
+    3: ("k_small", "-", "-", "-"),
 }
 
 
@@ -360,8 +361,10 @@ def main():
     names = STAGES[route]
 
     def dominant(pr):
-        stages = dict(zip(names, (pr["ms_prologue"], pr["ms_filter"], pr["ms_sweep"], pr["ms_finalize"])))
-        stages.pop("-", None)
+        stages = {}
+        for nm, v in zip(names, (pr["ms_prologue"], pr["ms_filter"], pr["ms_sweep"], pr["ms_finalize"])):
+            if nm != "-":
+                stages[nm] = v
         name = max(stages, key=stages.get)
         return name, stages[name] / pr["calls"], {k: v / pr["calls"] for k, v in stages.items()}
 
@@ -396,7 +399,7 @@ def main():
                "sample": f"the first {inst} of {w.B} instances of {w.name}, sweep_window (sort + one pass), {dt:.1f} s wall"}
 
     result = {"selections_per_s": world * w.B / (ms_step * 1e-3), "early_stop": route == 1,
-              "route": {0: "segment sweep", 1: "filter", 2: "buckets"}[route],
+              "route": {0: "segment sweep", 1: "filter", 2: "buckets", 3: "one launch"}[route],
               "examined_fraction": examined / nts, "input_copies": copies,
               "value_counts": "all n*R*B timestamps of the batch per call (nominal: the early stop examines examined_fraction of them; "
                               "full_sweep.value counts examined timestamps only)",

@@ -43,7 +43,7 @@ struct zl_handle {
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round, opt_cluster, opt_filter_stages, opt_checks_off, opt_filter_bulk, opt_tail_cap, opt_max_rounds;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round, opt_cluster, opt_filter_stages, opt_checks_off, opt_filter_bulk, opt_tail_cap, opt_max_rounds, opt_no_small;
     int epoch;               // calls so far: the two sets of per-call flags alternate
     int last_cuda_error;
     int launches;
@@ -80,6 +80,14 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     zl::FilterBufs fb = q.fb;
     if (!filter && !sumfast) memset(&fb, 0, sizeof(fb));
     if (ev) cudaEventRecord(ev[0], st);
+    if constexpr (!arith) {
+        if (q.small) {
+            // a few thousand timestamps an instance: everything in one kernel
+            zl::enqueue_small(q, p, st, src);
+            if (ev) for (int k = 1; k < PROF_EVENTS; ++k) cudaEventRecord(ev[k], st);
+            return;
+        }
+    }
     if (filter) zl::enqueue_range_head(q, fb, st, src);
     else zl::enqueue_prologue(q, fb, st, src);
     if constexpr (!arith) if (q.flags & ZL_FLAG_CHECK_SORTED) zl::enqueue_check_sorted(q, st);
@@ -118,6 +126,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
 cudaError_t raise_shared_memory_limits() {
     cudaError_t e = zl::prologue_limits();
     if (e == cudaSuccess) e = zl::range_limits();
+    if (e == cudaSuccess) e = zl::small_limits();
     if (e == cudaSuccess) e = zl::filter_limits();
     if (e == cudaSuccess) e = zl::heavy_limits();
     if (e == cudaSuccess) e = zl::range_rest_limits();
@@ -158,6 +167,13 @@ LaunchPlan make_plan(const zl_handle *h, int B) {
     long long target_rest = (long long)n * std::max(p.G_rest, 4) * rf / 100;
     target_rest = std::min<long long>(target_rest, (long long)p.cap * 4);
     p.target_rest = (int)std::max<long long>(target_rest, 32);
+    // the one-launch route: about eight timestamps a thread
+    p.threads_small = std::max(64, std::min(512, pow2_ceil((int)std::min<long long>(N / 8, 512))));
+    p.G_small = h->opt_lanes ? std::min(h->opt_lanes, p.threads_small) : std::max(1, std::min(32, pow2_floor(std::max(1, p.threads_small / n))));
+    long long target_small = (long long)n * std::max(p.G_small, 4) * rf / 100;
+    if (h->cfg.objective == ZL_OBJ_SUM) target_small = std::min<long long>(target_small, (long long)p.cap * 45 / 100);
+    target_small = std::min<long long>(target_small, (long long)p.cap * 4);
+    p.target_small = (int)std::max<long long>(target_small, 32);
     return p;
 }
 
@@ -412,6 +428,8 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
     } else if (!strcmp(key, "filter_bulk")) {
         if (value > 2) return ZL_ERR_INVALID_ARG;
         h->opt_filter_bulk = value;
+    } else if (!strcmp(key, "no_small")) {
+        h->opt_no_small = value != 0;               // small instances take the route larger ones would (bucket route)
     } else if (!strcmp(key, "max_rounds")) {
         h->opt_max_rounds = value;                  // the segment sweep gives up (ZL_ERR_TIMEOUT) after this many rounds of a segment
     } else if (!strcmp(key, "tail_cap")) {
@@ -443,14 +461,24 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
 }
 
 size_t zl_workspace_bytes(const zl_handle *h) { return h ? h->ws_bytes + h->staging_bytes : 0; }
+// The one-launch route: instances of at most SMALL_MAX timestamps in batches of a few per SM (a CTA an instance, all
+// resident at once: the call takes as long as one instance does), unless the handle asks for another route.  Larger
+// batches of small instances get more out of the bucket route's kernels.
+static bool small_route(const zl_handle *h) {
+    return (long long)h->cfg.n_workers * h->cfg.lookahead_R <= zl::SMALL_MAX && h->cfg.max_batch <= 4 * std::max(1, h->num_sms) &&
+           !h->opt_no_filter && !h->opt_no_small && !(h->cfg.flags & ZL_FLAG_FORCE_FILTER);
+}
+
 int32_t zl_launches_per_call(const zl_handle *h) {
     if (!h) return 0;
+    if (small_route(h)) return 1;
     const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter && h->fb.table != nullptr;
     const bool sumfast = !filter && !h->opt_no_filter && h->fb.scap != 0;
     return (filter ? (range_rest_split(h->cfg.n_workers, h->cfg.lookahead_R) ? 9 : 4) : 3) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
 }
 int32_t zl_route(const zl_handle *h) {
     if (!h || h->opt_no_filter) return 0;
+    if (small_route(h)) return 3;
     if (h->cfg.objective == ZL_OBJ_RANGE && h->fb.table != nullptr) return 1;
     return h->fb.scap != 0 ? 2 : 0;
 }
@@ -479,7 +507,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
     if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
     q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
-    q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds;
+    q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds; q.small = small_route(h) ? 1 : 0;
     if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
         uint32_t *base = h->fb.flags;
         q.fb.flags = base + 8 * (h->epoch & 1);
@@ -572,7 +600,7 @@ zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const i
         q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
         if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
         q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
-        q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds;
+        q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds; q.small = small_route(h) ? 1 : 0;
         if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
             uint32_t *base = h->fb.flags;
             q.fb.flags = base + 8 * (h->epoch & 1);
@@ -698,7 +726,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
     q.meta = meta; q.seg = seg; q.nres = p.nseg;
     memset(&q.fb, 0, sizeof(q.fb));
-    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0; q.cluster = q.filter_stages = 0; q.checks_off = 0; q.filter_bulk = 0; q.tail_cap = 0; q.rest_per_sm = 0; q.max_rounds = 0;
+    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0; q.cluster = q.filter_stages = 0; q.checks_off = 0; q.filter_bulk = 0; q.tail_cap = 0; q.rest_per_sm = 0; q.max_rounds = 0; q.small = (long long)n_workers * lookahead_R <= zl::SMALL_MAX && B <= 4 * std::max(1, tmp.num_sms) ? 1 : 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr, zl::MatBatch{d_ts});
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;

@@ -18,6 +18,7 @@ inline int pow2_ceil(int x) { int p = 1; while (p < x) p *= 2; return p; }
 struct LaunchPlan {
     int threads, G, nseg, cap, target; size_t smem;
     int G_rest, target_rest;                                      // lanes per row and round size when a CTA of 512 threads runs the sweep
+    int threads_small, G_small, target_small;                     // the same for the one-launch route of small instances
 };
 
 // Everything one call enqueues, for both the handle-based and the fixed-scratch entry points.
@@ -30,6 +31,7 @@ struct Pipeline {
     int prologue_threads, tail_threads;                           // 0: automatic
     int cluster, filter_stages, filter_bulk;                      // 0: automatic (cluster: CTAs per instance of k_range_head; filter_bulk: 1 copy engine, 2 per-lane copies)
     int tail_cap;                                                 // 0: default; else survivors the finishing CTA of the filter kernel has room for
+    int small;                                                    // 1: the one-launch route (instances of a few thousand timestamps)
     int max_rounds;                                               // 0: automatic; else the segment sweep's round limit
     int rest_per_sm;                                              // CTAs of k_range_rest resident per SM (0: ask the runtime)
     int checks_off;                                               // debug handle: unchecked kernels, clock stamps still taken
@@ -91,6 +93,10 @@ cudaError_t range_rest_limits();
 // sum_route.cu: the bucket route (plan, index pass, bucket kernel); `mid` is recorded before the bucket kernel
 void enqueue_bucket_route(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid);
 cudaError_t bucket_route_limits();
+
+// small.cu: the whole search for small instances in one launch
+void enqueue_small(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, const MatBatch &src);
+cudaError_t small_limits();
 
 // sweep.cu: the segment sweep (fallback of the fast routes, or the whole search) and K5
 void enqueue_sweep(const Pipeline &q, const FilterBufs &fb, const LaunchPlan &p, bool fast, cudaStream_t st, const MatBatch &src);

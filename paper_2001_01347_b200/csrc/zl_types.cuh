@@ -147,6 +147,7 @@ __device__ __forceinline__ uint32_t cell_of(uint32_t T, uint32_t cscale) { retur
 // Instances with at most this many survivors of the filter pass are finished by one CTA (k_tail);
 // larger ones go through cell scan, refinement and the bucket sweep.
 constexpr uint32_t TAIL_CAP = 2048;
+constexpr long long SMALL_MAX = 4096;    // instances of at most this many timestamps take the one-launch route
 __device__ __forceinline__ bool tail_instance(const InstMeta &M, const FilterBufs &F) { return M.count <= (uint32_t)F.tailcap; }
 
 }  // namespace zl

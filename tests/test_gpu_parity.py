@@ -312,7 +312,9 @@ def test_host_detected_errors():
         h.select_batched(ts)             # B > max_batch
     with pytest.raises(zl.ZipLineError):
         h.set_option("no_such_option", 1)
-    assert h.launches_per_call == 5 and h.workspace_bytes > 0      # tiny shape: prologue, plan, buckets, sweep, finalize
+    assert h.launches_per_call == 1 and h.workspace_bytes > 0      # tiny shape: one kernel does everything
+    h.set_option("no_small", 1)
+    assert h.launches_per_call == 5                                  # ... or the bucket route: prologue, plan, buckets, sweep, finalize
     h2 = zl.ZipLine(64, 128, 2)
     assert h2.launches_per_call == 4                                 # the filter route: head, filter, tail, one last kernel
     h2.destroy()
@@ -408,9 +410,11 @@ def test_mixed_batch_of_routes():
 
 
 # ---------------------------------------------------------------- the SUM routes
-def _sum_routes(ts_np):
+def _sum_routes(ts_np, options=None):
     B, n, R = ts_np.shape
     h = zl.ZipLine(n, R, B, 1)
+    for k, v in (options or {}).items():
+        h.set_option(k, v)
     sel = h.select_batched(torch.from_numpy(ts_np).cuda())
     torch.cuda.synchronize()
     buckets, tiles, overflow = h.filter_counts(B)
@@ -422,7 +426,7 @@ def _sum_routes(ts_np):
 def test_sum_routes_are_all_exercised_and_exact():
     # one bucket: the whole instance fits a shared-memory batch
     ts = zi.generate(zi.CONFIGS["c2"].with_(B=5, n=24, R=100))
-    got, buckets, tiles, overflow = _sum_routes(ts)
+    got, buckets, tiles, overflow = _sum_routes(ts, {"no_small": 1})
     assert (buckets == 1).all() and (tiles == 1).all() and (overflow == 0).all()
     assert_same(ts, 1, got)
     # several tiles of buckets, ragged last tile, rows of very different speeds
@@ -469,16 +473,34 @@ def test_sum_buckets_with_heavy_ties_and_odd_shapes():
         assert_same(ts, 1, got)
 
 
-def test_range_single_bucket_route_shapes():
-    # RANGE instances of at most 4096 timestamps are sorted whole by one CTA
+@pytest.mark.parametrize("objective", OBJ)
+def test_small_instances_one_launch_and_single_bucket_routes(objective):
+    # instances of at most 4096 timestamps: one kernel does the whole search (route 3); with that route off they are
+    # sorted whole by one CTA of the bucket route (route 2)
     rng = np.random.default_rng(99)
-    for n, R, B, hi in ((16, 64, 300, 10 ** 5), (4096, 1, 2, 1000), (1, 4096, 2, 50), (63, 65, 5, 7), (2, 2048, 3, 10 ** 9)):
+    for n, R, B, hi in ((16, 64, 300, 10 ** 5), (4096, 1, 2, 1000), (1, 4096, 2, 50), (63, 65, 5, 7), (2, 2048, 3, 10 ** 9), (1, 1, 3, 5)):
         inc = rng.integers(0, hi, size=(B, n, R))
         ts = (rng.integers(0, 3 * hi, size=(B, n, 1)) + np.cumsum(inc, axis=2)).astype(np.int64)
-        h = zl.ZipLine(n, R, B, 0)
+        h = zl.ZipLine(n, R, B, objective)
+        assert h.route == 3 and h.launches_per_call == 1
+        h.set_option("no_small", 1)
         assert h.route == 2
         h.destroy()
-        assert_same(ts, 0, gpu_select(ts, 0))
+        h = zl.ZipLine(n, R, 5000, objective)                # a batch of thousands: the bucket route
+        assert h.route == 2
+        h.destroy()
+        assert_same(ts, objective, gpu_select(ts, objective))
+        assert_same(ts, objective, gpu_select(ts, objective, options={"no_small": 1}))
+    # errors per instance come out of the one kernel too
+    ts = np.cumsum(np.ones((3, 4, 6), dtype=np.int64), axis=2) * 10
+    ts[1, 2, 3] = 5
+    ts[2, 0, 0] = -4
+    idx, barrier, wait, status = gpu_select(ts, objective, flags=zl.ZL_FLAG_CHECK_SORTED)
+    assert status.tolist() == [0, zl.binding.ZL_ERR_UNSORTED, zl.binding.ZL_ERR_INVALID_ARG]
+    assert (idx[1:] == -1).all() and (barrier[1:] == np.iinfo(np.int64).min).all()
+
+
+def test_range_filter_route_starts_above_the_small_sizes():
     h = zl.ZipLine(64, 65, 1, 0)
     assert h.route == 1                        # 4160 timestamps: the filter route
     h.destroy()
