@@ -1,7 +1,8 @@
 // The RANGE filter pass (k_filter on stored rows, k_filter_arith on predicted rows) and k_tail, which finishes
-// the instances that are left with few survivors: the kernels every handle runs unless it asks for the checked
-// ones (range_filter.cu).
+// the instances that are left with few survivors.  Each has an instantiation that tests its indices (CHECK), which a
+// handle created with ZL_FLAG_DEBUG_CHECKS runs.
 #include "zl_batch.cuh"
+#include "zl_guard.cuh"
 #include "zl_host.h"
 
 namespace zl {
@@ -16,20 +17,24 @@ constexpr int FILTER_STAGES = 3;      // ring slots per warp
 constexpr int FILTER_CHUNK = 256;     // timestamps per slot (FILTER_CHUNK / 64 16-byte copies per lane)
 constexpr int FILTER_SLOT = FILTER_CHUNK + 2;   // + the successor of the slot's last element, + padding
 
+template <bool CHECK>
 struct FilterCtx {
     const uint32_t *tab; uint64_t *list; uint32_t *cellmax; unsigned int *scount;
     uint32_t cscale, fscale, lmin, regcap, dmin;
+    uint32_t cells, fcells;
+    Guard<CHECK> g;               // CHECK: table, list and cell indices are tested before they are used
 };
 
 // Table test of the (up to) two elements of a lane, warp-aggregated append of the survivors.
-__device__ __forceinline__ void filter_pair(const FilterCtx &c, int lane, bool va, uint32_t Ta, uint32_t na,
+template <bool CHECK>
+__device__ __forceinline__ void filter_pair(const FilterCtx<CHECK> &c, int lane, bool va, uint32_t Ta, uint32_t na,
                                             bool vb, uint32_t Tb, uint32_t nb) {
     // cheap necessary condition first: most elements belong to fast workers and stop here
     bool ka = va && Ta <= c.lmin && na - Ta > c.dmin;
     bool kb = vb && Tb <= c.lmin && nb - Tb > c.dmin;
     if (!__any_sync(FULL, ka || kb)) return;
-    if (ka) ka = na > max(Ta, c.tab[cell_of(Ta, c.cscale)]);
-    if (kb) kb = nb > max(Tb, c.tab[cell_of(Tb, c.cscale)]);
+    if (ka) { const uint32_t cc = cell_of(Ta, c.cscale); ka = c.g.ok(cc, c.cells, ACC_TAB) && na > max(Ta, c.tab[cc]); }
+    if (kb) { const uint32_t cc = cell_of(Tb, c.cscale); kb = c.g.ok(cc, c.cells, ACC_TAB) && nb > max(Tb, c.tab[cc]); }
     const unsigned ma = __ballot_sync(FULL, ka), mb = __ballot_sync(FULL, kb);
     if ((ma | mb) == 0) return;
     const int na_cnt = __popc(ma), tot = na_cnt + __popc(mb);
@@ -40,19 +45,22 @@ __device__ __forceinline__ void filter_pair(const FilterCtx &c, int lane, bool v
     if (ka) {
         const unsigned pos = base + __popc(ma & below);
         if (pos < c.regcap) c.list[pos] = ((uint64_t)Ta << 32) | na;
-        atomicMax(&c.cellmax[cell_of(Ta, c.fscale)], na);
+        const uint32_t fc = cell_of(Ta, c.fscale);
+        if (c.g.ok(fc, c.fcells, ACC_CELLMAX)) atomicMax(&c.cellmax[fc], na);
     }
     if (kb) {
         const unsigned pos = base + na_cnt + __popc(mb & below);
         if (pos < c.regcap) c.list[pos] = ((uint64_t)Tb << 32) | nb;
-        atomicMax(&c.cellmax[cell_of(Tb, c.fscale)], nb);
+        const uint32_t fc = cell_of(Tb, c.fscale);
+        if (c.g.ok(fc, c.fcells, ACC_CELLMAX)) atomicMax(&c.cellmax[fc], nb);
     }
 }
 
 // The 64 elements of a slot starting at `off`: element pairs per lane, successor of the pair from the
 // slot itself (the element after the slot's last one sits right behind it).  Returns the time of the
 // last valid element handled by lane 31 (0xffffffff past the row's end).
-__device__ __forceinline__ uint32_t filter_half(const FilterCtx &C, const int64_t *slot, int off, int i0, int lim, int R,
+template <bool CHECK>
+__device__ __forceinline__ uint32_t filter_half(const FilterCtx<CHECK> &C, const int64_t *slot, int off, int i0, int lim, int R,
                                                 uint32_t tminlo, int lane) {
     const int i = i0 + off + 2 * lane;
     const bool va = i < lim, vb = i + 1 < lim;                    // lim: end of what was requested of the row (<= R)
@@ -66,7 +74,8 @@ __device__ __forceinline__ uint32_t filter_half(const FilterCtx &C, const int64_
 
 // 128 timestamps of a slot, with the one after them, that lie inside the row: no bounds checks, one vote
 // for all four elements of a lane.  Returns the time of the last of the 128.
-__device__ __forceinline__ uint32_t filter_slot_inside(const FilterCtx &C, const int64_t *slot, uint32_t tminlo, int lane) {
+template <bool CHECK>
+__device__ __forceinline__ uint32_t filter_slot_inside(const FilterCtx<CHECK> &C, const int64_t *slot, uint32_t tminlo, int lane) {
     const longlong2 p0 = *reinterpret_cast<const longlong2 *>(slot + 2 * lane);
     const longlong2 p1 = *reinterpret_cast<const longlong2 *>(slot + 64 + 2 * lane);
     const uint32_t a0 = (uint32_t)(uint64_t)p0.x - tminlo, b0 = (uint32_t)(uint64_t)p0.y - tminlo;
@@ -81,14 +90,18 @@ __device__ __forceinline__ uint32_t filter_slot_inside(const FilterCtx &C, const
     return __shfl_sync(FULL, b1, 31);
 }
 
-__global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R, int flags, int rows_per_cta, int req_round,
+template <bool CHECK>
+__global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R, int B, int flags, int rows_per_cta, int req_round,
                                                   InstMeta *meta, FilterBufs F) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ unsigned int scount;
     const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
     const InstMeta M = meta[b];
+    const Guard<CHECK> gd{F.dbg, (uint32_t)(b * gridDim.x + blockIdx.x)};
     uint32_t *rc = F.rcnt + (size_t)b * F.nreg + blockIdx.x;
+    if (!gd.ok((size_t)b * F.nreg + blockIdx.x, (size_t)B * F.nreg, ACC_RCNT) ||
+        !gd.ok((size_t)b * F.list1cap + ((size_t)blockIdx.x + 1) * F.regcap - 1, (size_t)B * F.list1cap, ACC_LIST)) return;
     if (M.status != ZL_OK || M.cscale == 0) { if (tid == 0) *rc = 0; return; }
     const uint32_t cells = (uint32_t)F.cells, lmin = (uint32_t)M.lmin;
     const uint32_t tminlo = (uint32_t)(uint64_t)M.tmin - 1u;     // relative time = low word of t - tminlo
@@ -99,10 +112,11 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
     if (tid == 0) scount = 0;
     __syncthreads();
     const bool full = (flags & ZL_FLAG_FULL_SWEEP) != 0;
-    FilterCtx C;
+    FilterCtx<CHECK> C;
     C.tab = tab; C.list = F.list1 + (size_t)b * F.list1cap + (size_t)blockIdx.x * F.regcap;
     C.cellmax = F.cellmax + (size_t)b * F.fcells; C.scount = &scount;
     C.cscale = M.cscale; C.fscale = M.fscale; C.lmin = lmin; C.regcap = (uint32_t)F.regcap; C.dmin = M.dmin;
+    C.cells = cells; C.fcells = (uint32_t)F.fcells; C.g = gd;
     const int r0 = blockIdx.x * rows_per_cta, r1 = min(r0 + rows_per_cta, n);
     const bool vec2 = (R % 2 == 0) && (((uintptr_t)ts & 15) == 0);
     const size_t rstride = (size_t)nw * R;                        // between consecutive rows of this warp
@@ -202,13 +216,17 @@ __global__ void __launch_bounds__(1024) k_filter(const int64_t *ts, int n, int R
 // element's own iteration is the row's interval, so a whole row whose interval does not exceed dmin is settled
 // at once (only its last element, whose next is infinite, can pass); the other rows are walked up to lmin, an
 // element per lane.  Same regions, lists and counters as k_filter.
-__global__ void __launch_bounds__(256) k_filter_arith(const AriBatch src, int n, int R, int rows_per_cta, InstMeta *meta, FilterBufs F) {
+template <bool CHECK>
+__global__ void __launch_bounds__(256) k_filter_arith(const AriBatch src, int n, int R, int B, int rows_per_cta, InstMeta *meta, FilterBufs F) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ unsigned int scount;
     const int b = blockIdx.y, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
     const InstMeta M = meta[b];
+    const Guard<CHECK> gd{F.dbg, (uint32_t)(b * gridDim.x + blockIdx.x)};
     uint32_t *rc = F.rcnt + (size_t)b * F.nreg + blockIdx.x;
+    if (!gd.ok((size_t)b * F.nreg + blockIdx.x, (size_t)B * F.nreg, ACC_RCNT) ||
+        !gd.ok((size_t)b * F.list1cap + ((size_t)blockIdx.x + 1) * F.regcap - 1, (size_t)B * F.list1cap, ACC_LIST)) return;
     if (M.status != ZL_OK || M.cscale == 0) { if (tid == 0) *rc = 0; return; }
     const uint32_t cells = (uint32_t)F.cells;
     uint32_t *tab = (uint32_t *)smem;
@@ -216,10 +234,11 @@ __global__ void __launch_bounds__(256) k_filter_arith(const AriBatch src, int n,
     for (uint32_t c = tid; c < cells; c += nt) tab[c] = tg[c];
     if (tid == 0) scount = 0;
     __syncthreads();
-    FilterCtx C;
+    FilterCtx<CHECK> C;
     C.tab = tab; C.list = F.list1 + (size_t)b * F.list1cap + (size_t)blockIdx.x * F.regcap;
     C.cellmax = F.cellmax + (size_t)b * F.fcells; C.scount = &scount;
     C.cscale = M.cscale; C.fscale = M.fscale; C.lmin = (uint32_t)M.lmin; C.regcap = (uint32_t)F.regcap; C.dmin = M.dmin;
+    C.cells = cells; C.fcells = (uint32_t)F.fcells; C.g = gd;
     const AriRows rows = src.inst(b, n, R);
     const int r0 = blockIdx.x * rows_per_cta, r1 = min(r0 + rows_per_cta, n);
     for (int r = r0 + warp; r < r1; r += nw) {
@@ -253,14 +272,16 @@ __global__ void __launch_bounds__(256) k_filter_arith(const AriBatch src, int n,
 // exclusive prefix maximum, drop every survivor whose next does not exceed the value at its cell's
 // start), then sorts what is left and sweeps it.  Dropped survivors never hold the running maximum
 // alone, so nothing has to be carried in.
-template <class SRC>
+template <class SRC, bool CHECK>
 __global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBufs F, int n, int nres, SegResult *seg, int tcap,
-                                                  const SRC src, int R, int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
+                                                  const SRC src, int R, int B, int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
     grid_dep_wait();
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ uint64_t tmp[34];
     __shared__ unsigned int sstatus, fill;
     const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+    const Guard<CHECK> gd{F.dbg, (uint32_t)b};
+    const int cells = F.cells;
     const InstMeta M = meta[b];
     if (tid == 0) {
         // tell the later kernels of this call whether they have anything to do
@@ -273,7 +294,6 @@ __global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBu
     uint32_t *g = (uint32_t *)smem;                               // [cells]
     Key<uint32_t> *keys = (Key<uint32_t> *)(smem + (size_t)F.cells * 4);
     const BatchWS<uint32_t> ws{keys, keys + tcap, (uint32_t *)(keys + 2 * (size_t)tcap), tcap};
-    const int cells = F.cells;
     for (int c = tid; c < cells; c += nt) g[c] = 0;
     if (tid == 0) { sstatus = 0; fill = 0; }
     __syncthreads();
@@ -281,8 +301,10 @@ __global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBu
         const uint32_t c = F.rcnt[(size_t)b * F.nreg + r];
         const uint64_t *src = F.list1 + (size_t)b * F.list1cap + (size_t)r * F.regcap;
         for (uint32_t i = lane; i < c; i += 32) {
+            if (!gd.ok((size_t)b * F.list1cap + (size_t)r * F.regcap + i, (size_t)B * F.list1cap, ACC_LIST)) continue;
             const uint64_t w = src[i];
-            atomicMax(&g[cell_of((uint32_t)(w >> 32), M.cscale)], (uint32_t)w);
+            const uint32_t cc = cell_of((uint32_t)(w >> 32), M.cscale);
+            if (gd.ok(cc, (uint64_t)cells, ACC_TAB)) atomicMax(&g[cc], (uint32_t)w);
         }
     }
     __syncthreads();
@@ -301,15 +323,17 @@ __global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBu
         const uint64_t *src = F.list1 + (size_t)b * F.list1cap + (size_t)r * F.regcap;
         for (uint32_t i0 = 0; i0 < c; i0 += 32) {
             const uint32_t i = i0 + lane;
-            const uint64_t w = i < c ? src[i] : 0ull;
+            const uint64_t w = (i < c && gd.ok((size_t)b * F.list1cap + (size_t)r * F.regcap + i, (size_t)B * F.list1cap, ACC_LIST)) ? src[i] : 0ull;
             const uint32_t T = (uint32_t)(w >> 32), nx = (uint32_t)w;
-            const bool keep = i < c && nx > max(T, g[cell_of(T, M.cscale)]);
+            const uint32_t cc = i < c ? cell_of(T, M.cscale) : 0u;
+            const bool keep = i < c && gd.ok(cc, (uint64_t)cells, ACC_TAB) && nx > max(T, g[cc]);
             const unsigned km = __ballot_sync(FULL, keep);
             if (km == 0) continue;
             unsigned base = 0;
             if (lane == 0) base = atomicAdd(&fill, (unsigned)__popc(km));
             base = __shfl_sync(FULL, base, 0);
-            if (keep) keys[base + __popc(km & ((1u << lane) - 1u))].w = w;
+            const unsigned pos = base + __popc(km & ((1u << lane) - 1u));
+            if (keep && gd.ok(pos, (uint64_t)tcap, ACC_KEYS)) keys[pos].w = w;
         }
     }
     __syncthreads();
@@ -323,13 +347,14 @@ __global__ void __launch_bounds__(1024, 1) k_tail(const InstMeta *meta, FilterBu
     const int fst = best.valid ? ZL_OK : ZL_ERR_TIMEOUT;          // a valid instance always has a candidate
     const int64_t bar = fst == ZL_OK ? M.tmin + (int64_t)(best.t - 1) + (int64_t)best.d : INT64_MIN;
     if (tid == 0) {
-        seg[(size_t)b * nres] = best;
+        if (gd.ok((size_t)b * nres, (size_t)B * nres, ACC_SEG)) seg[(size_t)b * nres] = best;
         wait[b] = fst == ZL_OK ? (int64_t)best.d : INT64_MIN;
         barrier[b] = bar;
         if (status) status[b] = fst;
     }
     for (int p = tid; p < n; p += nt)
-        idx[(size_t)b * n + p] = fst == ZL_OK ? last_index_not_after(src.inst(b, n, R).row(p), R, bar) : -1;
+        if (gd.ok((size_t)b * n + p, (size_t)B * n, ACC_IDX))
+            idx[(size_t)b * n + p] = fst == ZL_OK ? last_index_not_after(src.inst(b, n, R).row(p), R, bar) : -1;
 }
 
 template <class SRC>
@@ -345,26 +370,38 @@ static void enqueue_filter_t(const Pipeline &q, FilterBufs &fb, cudaStream_t st,
     fb.nreg = (int)((q.n + rpc - 1) / rpc);
     fb.regcap = fb.list1cap / fb.nreg;
     const size_t fsmem = (size_t)fb.cells * 4 + (size_t)nw * FILTER_STAGES * FILTER_SLOT * 8;
-    if constexpr (arith)
-        launch_dep(!((q.pdl_off >> 1) & 1), k_filter_arith, dim3(fb.nreg, q.B), dim3(threads), (size_t)fb.cells * 4, st, src, q.n, q.R, (int)rpc, q.meta, fb);
-    else
-        launch_dep(!((q.pdl_off >> 1) & 1), k_filter, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.flags, (int)rpc, q.filter_round ? q.filter_round : 8, q.meta, fb);
+    // a debug handle runs the instantiations that test their indices
+    const bool check = (q.flags & ZL_FLAG_DEBUG_CHECKS) && fb.dbg && !q.checks_off;
+    if constexpr (arith) {
+        if (check) launch_dep(!((q.pdl_off >> 1) & 1), k_filter_arith<true>, dim3(fb.nreg, q.B), dim3(threads), (size_t)fb.cells * 4, st, src, q.n, q.R, q.B, (int)rpc, q.meta, fb);
+        else launch_dep(!((q.pdl_off >> 1) & 1), k_filter_arith<false>, dim3(fb.nreg, q.B), dim3(threads), (size_t)fb.cells * 4, st, src, q.n, q.R, q.B, (int)rpc, q.meta, fb);
+    } else {
+        if (check) launch_dep(!((q.pdl_off >> 1) & 1), k_filter<true>, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.B, q.flags, (int)rpc, q.filter_round ? q.filter_round : 8, q.meta, fb);
+        else launch_dep(!((q.pdl_off >> 1) & 1), k_filter<false>, dim3(fb.nreg, q.B), dim3(threads), fsmem, st, q.ts, q.n, q.R, q.B, q.flags, (int)rpc, q.filter_round ? q.filter_round : 8, q.meta, fb);
+    }
     if (mid) cudaEventRecord(mid, st);
     // instances with at most tcap survivors are finished by one CTA each; with many instances a smaller limit lets more
     // of those CTAs share an SM
     const int tcap = (int)std::min<long long>(many ? (long long)TAIL_CAP / 2 : (long long)TAIL_CAP, pow2_ceil(std::max(64, fb.list1cap)));
     fb.tailcap = tcap;
-    launch_dep(!((q.pdl_off >> 2) & 1), k_tail<SRC>, dim3(q.B), dim3(q.tail_threads ? q.tail_threads : many ? (tcap <= 1024 ? 128 : 256) : std::max(64, std::min(1024, tcap / 2))), (size_t)tcap * 20 + (size_t)fb.cells * 4, st,
-               (const InstMeta *)q.meta, fb, q.n, q.nres, q.seg, tcap, src, q.R, q.idx, q.barrier, q.wait, q.status);
+    const int tthreads = q.tail_threads ? q.tail_threads : many ? (tcap <= 1024 ? 128 : 256) : std::max(64, std::min(1024, tcap / 2));
+    const size_t tsmem = (size_t)tcap * 20 + (size_t)fb.cells * 4;
+    if (check) launch_dep(!((q.pdl_off >> 2) & 1), k_tail<SRC, true>, dim3(q.B), dim3(tthreads), tsmem, st,
+                          (const InstMeta *)q.meta, fb, q.n, q.nres, q.seg, tcap, src, q.R, q.B, q.idx, q.barrier, q.wait, q.status);
+    else launch_dep(!((q.pdl_off >> 2) & 1), k_tail<SRC, false>, dim3(q.B), dim3(tthreads), tsmem, st,
+                    (const InstMeta *)q.meta, fb, q.n, q.nres, q.seg, tcap, src, q.R, q.B, q.idx, q.barrier, q.wait, q.status);
 }
 
 void enqueue_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid, const MatBatch &src) { enqueue_filter_t(q, fb, st, mid, src); }
 void enqueue_filter(const Pipeline &q, FilterBufs &fb, cudaStream_t st, cudaEvent_t mid, const AriBatch &src) { enqueue_filter_t(q, fb, st, mid, src); }
 
 cudaError_t filter_limits() {
-    cudaError_t e = cudaFuncSetAttribute(k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tail<MatBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tail<AriBatch>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(k_filter<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_filter<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tail<MatBatch, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tail<AriBatch, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tail<MatBatch, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tail<AriBatch, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
     return e;
 }
 

@@ -94,9 +94,8 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
     if (ev) cudaEventRecord(ev[1], st);
     if (filter) {
         // the filter kernel, then everything it left undone and the outputs in one more launch
-        const bool checked = ((q.flags & ZL_FLAG_DEBUG_CHECKS) && !q.checks_off) || q.filter_bulk;
-        if (checked) {
-            // the self-checking variants of the two kernels (also the ones with the bulk-copy ring)
+        if (q.filter_bulk) {
+            // on request: the variant of the two kernels whose rows arrive through a ring filled by the copy engine
             zl::enqueue_range_filter(q, fb, st, src);
             if (ev) cudaEventRecord(ev[2], st);
             zl::enqueue_range_tail(q, fb, st, src);

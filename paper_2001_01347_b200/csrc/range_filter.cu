@@ -32,6 +32,7 @@
 #include <cooperative_groups.h>
 
 #include "zl_batch.cuh"
+#include "zl_guard.cuh"
 #include "zl_host.h"
 
 namespace cg = cooperative_groups;
@@ -45,22 +46,6 @@ struct RangeParams {
     uint32_t *dbg;                       // CHECK: [0] code of the first violation, [1] its CTA, [2..3] the index
     unsigned long long *stamps;          // debug handles: [ctas][16] nanosecond clock at the phase boundaries of every CTA
     uint32_t smem_bytes, ctas;           // of the kernel at hand
-};
-
-enum RangeAccess : int {
-    ACC_PART = 1, ACC_PTAB, ACC_RCNT, ACC_LIST, ACC_CELLMAX, ACC_BCNT, ACC_META, ACC_SEG, ACC_IDX,
-    ACC_COPY_SRC, ACC_COPY_DST, ACC_COPY_ALIGN, ACC_TAB, ACC_ARR, ACC_COLS, ACC_REQS, ACC_SLOT, ACC_KEYS
-};
-
-template <bool CHECK>
-struct Guard {
-    uint32_t *dbg; uint32_t cta;
-    __device__ __forceinline__ bool ok(uint64_t i, uint64_t lim, int code) const {
-        if (!CHECK) return true;
-        if (i < lim) return true;
-        if (atomicCAS(&dbg[0], 0u, (uint32_t)code) == 0u) { dbg[1] = cta; dbg[2] = (uint32_t)i; dbg[3] = (uint32_t)(i >> 32); }
-        return false;
-    }
 };
 
 __device__ __forceinline__ unsigned long long global_ns() {

@@ -105,6 +105,24 @@ def test_filter_route_on_tiny_shapes_vs_enumerator(regime, checked):
         h.destroy()
 
 
+@pytest.mark.parametrize("variant", [1, 2])
+def test_filter_ring_variants_are_exact(variant):
+    # the filter pass whose rows arrive through a shared-memory ring filled by the copy engine (bulk copies counted on
+    # mbarriers, 1) or by 16-byte copies of every lane (2): slower than the default kernels on these workloads, kept as
+    # options, and exact
+    for w in (zi.CONFIGS["c4"].with_(B=6, n=200, R=700), zi.CONFIGS["c3"].with_(B=40), zi.CONFIGS["c2"].with_(B=30, n=100, R=150)):
+        ts = zi.generate(w)
+        for flags in (0, zl.ZL_FLAG_DEBUG_CHECKS, zl.ZL_FLAG_FULL_SWEEP):
+            h = zl.ZipLine(w.n, w.R, w.B, 0, 0, flags)
+            h.set_option("filter_bulk", variant)
+            sel = h.select_batched(torch.from_numpy(ts).cuda())
+            torch.cuda.synchronize()
+            assert_same(ts, 0, (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()))
+            if flags & zl.ZL_FLAG_DEBUG_CHECKS:
+                assert h.debug_report() == (0, 0, 0) and h.check_canaries()[1] == 0
+            h.destroy()
+
+
 def test_filter_route_dense_ties_just_above_the_single_batch_size():
     # 256 instances of slightly more than 4096 timestamps with many equal values: the filter route's natural smallest shapes
     rng = np.random.default_rng(301)
