@@ -47,7 +47,9 @@ __global__ void __launch_bounds__(REST_THREADS) k_range_rest(const SRC src, cons
     unsigned long long *stamps = F.dbg && (int)blockIdx.x < F.maxctas ? (unsigned long long *)(F.dbg + 16) + (size_t)blockIdx.x * 16 : nullptr;
 #define ZL_STAMP(k) do { if (stamps && threadIdx.x == 0) { unsigned long long t_; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t_)); stamps[k] = t_; } } while (0)
     ZL_STAMP(6);
-    const RowEnds first = finalize_first_ends(src, P.B, P.n, P.R);  // input: no need to wait for it
+    const RowEnds first = finalize_first_ends(src, P.B, P.n, P.R);
+    // (Input, read before the wait: this is not the call's first kernel, and it starts only when every CTA of its predecessor
+    // has exited, i.e. has passed its own wait, so whatever produced the input before the call had completed by then.)
     grid_dep_wait();
     ZL_STAMP(7);
     extern __shared__ __align__(16) unsigned char smem[];

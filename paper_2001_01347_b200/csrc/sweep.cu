@@ -20,7 +20,9 @@ template <class SRC>
 __global__ void __launch_bounds__(256) k_finalize(const SRC src, int B, int n, int R, int nseg, FilterBufs F, int nres,
                                                   int objective, int filter, const InstMeta *meta, const SegResult *seg,
                                                   int32_t *idx, int64_t *barrier, int64_t *wait, int32_t *status) {
-    const RowEnds first = finalize_first_ends(src, B, n, R);      // input: no need to wait for it
+    const RowEnds first = finalize_first_ends(src, B, n, R);
+    // (Input, read before the wait: this is not the call's first kernel, and it starts only when every CTA of its predecessor
+    // has exited, i.e. has passed its own wait, so whatever produced the input before the call had completed by then.)
     grid_dep_wait();
     if (filter == 1 && F.flags[2] == 0) return;                   // the tail kernel finished every instance of the call
     finalize_all(src, B, n, R, nseg, F, nres, objective, filter, meta, seg, idx, barrier, wait, status, 0u, &first);

@@ -254,8 +254,8 @@ __device__ void sweep_items(const SweepParams &P, const SRC &src, SweepShared &s
 // per lane; the warp of the instance's first rows also writes wait, barrier and status.
 // filter: 0 only the segment sweep ran, 1 the RANGE filter route (an instance with few survivors has one result, left
 // by the filter kernel), 2 the bucket route.  `forced`: a status that overrides the instance's own when not ZL_OK.
-// `pre`: the first and last element of the lane's row when the caller loaded them already (they are input, so that can
-// happen before the kernel's predecessors are done), else nullptr.
+// `pre`: the first and last element of the lane's row when the caller loaded them already (they are input: a kernel that
+// is not the first of its call may read them before it waits for its predecessor), else nullptr.
 struct RowEnds { int64_t e0, eR; };
 // An instance's record and its first partial result, for a caller that loads them ahead of the call.
 struct FirstResult { InstMeta M; uint64_t d, t; unsigned long long vs; };
