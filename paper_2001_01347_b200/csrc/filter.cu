@@ -58,7 +58,7 @@ __device__ __forceinline__ void filter_pair(const FilterCtx<CHECK> &c, int lane,
 
 // The 64 elements of a slot starting at `off`: element pairs per lane, successor of the pair from the
 // slot itself (the element after the slot's last one sits right behind it).  Returns the time of the
-// last valid element handled by lane 31 (0xffffffff past the row's end).
+// last of them that belongs to the request.
 template <bool CHECK>
 __device__ __forceinline__ uint32_t filter_half(const FilterCtx<CHECK> &C, const int64_t *slot, int off, int i0, int lim, int R,
                                                 uint32_t tminlo, int lane) {
@@ -69,7 +69,10 @@ __device__ __forceinline__ uint32_t filter_half(const FilterCtx<CHECK> &C, const
     const uint32_t Tb = vb ? (uint32_t)(uint64_t)ab.y - tminlo : 0xffffffffu;
     const uint32_t nb = i + 2 < R ? (uint32_t)(uint64_t)slot[off + 2 * lane + 2] - tminlo : 0xffffffffu;
     filter_pair(C, lane, va, Ta, Tb, vb, Tb, nb);
-    return __shfl_sync(FULL, Tb, 31);
+    // the last of the 64 that belongs to the request (the caller passes at least one): whether the row has passed lmin is
+    // decided by a real element, never by the filler behind the request's end
+    const int last = min(63, lim - 1 - (i0 + off));
+    return __shfl_sync(FULL, (last & 1) ? Tb : Ta, last >> 1);
 }
 
 // 128 timestamps of a slot, with the one after them, that lie inside the row: no bounds checks, one vote

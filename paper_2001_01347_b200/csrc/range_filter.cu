@@ -97,8 +97,7 @@ __device__ __forceinline__ uint32_t filter_128(const FCtx<CHECK> &C, const int64
 }
 
 // 64 timestamps starting at slot[off] = element i0 + off of the row, of which those below `lim` count; the
-// successor of the row's last element is infinite.  Returns the time lane 31's second element has
-// (0xffffffff past the end).
+// successor of the row's last element is infinite.  Returns the time of the last of them that belongs to the request.
 template <bool CHECK>
 __device__ __forceinline__ uint32_t filter_64(const FCtx<CHECK> &C, const int64_t *slot, int off, int i0, int lim, int R, int lane) {
     const int i = i0 + off + 2 * lane;
@@ -110,7 +109,8 @@ __device__ __forceinline__ uint32_t filter_64(const FCtx<CHECK> &C, const int64_
     const uint32_t nb = i + 2 < R ? (uint32_t)(uint64_t)slot[off + 2 * lane + 2] - C.tminlo : 0xffffffffu;
     if (va && Ta <= C.lmin && na - Ta > C.dmin) filter_candidate(C, Ta, na);
     if (vb && Tb <= C.lmin && nb - Tb > C.dmin) filter_candidate(C, Tb, nb);
-    return __shfl_sync(FULL, Tb, 31);
+    const int last = min(63, lim - 1 - (i0 + off));               // the last of the 64 that belongs to the request
+    return __shfl_sync(FULL, (last & 1) ? Tb : Ta, last >> 1);
 }
 
 // Elements j0, j0 + 1, ... of a row by plain loads (rows that cannot take bulk copies, and the rare row whose
@@ -174,7 +174,7 @@ __device__ __forceinline__ void filter_pair(const FCtx<CHECK> &c, int lane, bool
 // Up to 128 timestamps of a slot starting at slot[off] = element i0 + off of the row, of which those below `lim` (the
 // end of what was requested of the row, <= R) count: lane l holds elements 2l, 2l + 1, 64 + 2l and 65 + 2l of them,
 // each one's successor from the slot itself (the element after the slot's last one sits right behind it; the row's
-// last element has none).  Returns the time of the last of the 128 (0xffffffff past the end of the request).
+// last element has none).  Returns the time of the last of them that belongs to the request.
 template <bool CHECK>
 __device__ __forceinline__ uint32_t filter_partial(const FCtx<CHECK> &C, const int64_t *slot, int off, int i0, int lim, int R, int lane) {
     const int i = i0 + off + 2 * lane;
@@ -196,7 +196,12 @@ __device__ __forceinline__ uint32_t filter_partial(const FCtx<CHECK> &C, const i
         okmask |= (i + 64 < lim ? 4u : 0u) | (i + 65 < lim ? 8u : 0u);
     }
     filter_quad(C, lane, T, nx, okmask);
-    return __shfl_sync(FULL, second ? T[3] : T[1], 31);
+    // the last of the 128 that belongs to the request (the caller passes at least one): whether the row has passed lmin is
+    // decided by a real element, never by the filler behind the request's end
+    const int last = min(127, lim - 1 - (i0 + off));
+    const int l64 = last & 63;
+    const uint32_t v = last >= 64 ? ((l64 & 1) ? T[3] : T[2]) : ((l64 & 1) ? T[1] : T[0]);
+    return __shfl_sync(FULL, v, l64 >> 1);
 }
 
 // 128 timestamps of a slot, with the one after them, that lie inside the row and the request: no bounds checks.

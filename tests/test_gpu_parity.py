@@ -123,6 +123,27 @@ def test_filter_ring_variants_are_exact(variant):
             h.destroy()
 
 
+@pytest.mark.parametrize("variant", [0, 1, 2])
+def test_filter_route_rows_far_from_arithmetic(variant):
+    # rows with rare long iterations among short ones: the number of a row's elements before the first exhausted row's
+    # end is then badly estimated from the row's end points, and the filter pass has to go on past what it asked for
+    rng = np.random.default_rng(302)
+    for n, R, B in ((64, 100, 40), (17, 257, 300), (513, 256, 9), (129, 257, 17), (300, 1025, 3)):
+        inc = np.where(rng.random((B, n, R)) < 0.02, 5000, rng.integers(1, 30, size=(B, n, R)))
+        ts = (rng.integers(0, 1000, size=(B, n, 1)) + np.cumsum(inc, axis=2)).astype(np.int64)
+        for flags in (0, zl.ZL_FLAG_DEBUG_CHECKS):
+            h = zl.ZipLine(n, R, B, 0, 0, flags)
+            assert h.route == 1
+            if variant:
+                h.set_option("filter_bulk", variant)
+            sel = h.select_batched(torch.from_numpy(ts).cuda())
+            torch.cuda.synchronize()
+            assert_same(ts, 0, (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()))
+            if flags:
+                assert h.debug_report() == (0, 0, 0) and h.check_canaries()[1] == 0
+            h.destroy()
+
+
 def test_filter_route_dense_ties_just_above_the_single_batch_size():
     # 256 instances of slightly more than 4096 timestamps with many equal values: the filter route's natural smallest shapes
     rng = np.random.default_rng(301)
