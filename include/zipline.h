@@ -6,8 +6,8 @@
  * e^p_1 <= ... <= e^p_R.  One element is picked per worker to form Z; the
  * waiting time is d_Z = max(Z) - min(Z); the selection returned is
  * Z* = argmin d_Z and the next synchronisation barrier is max(Z*).  When
- * several Z reach the minimum the earliest barrier is taken (Fig. 3 caption,
- * "the first minimum d_Z is selected").
+ * several Z reach the minimum the earliest barrier is taken (Fig. 3's caption
+ * says that of equal minima the first one found wins).
  *
  * Every entry point is extern "C", takes plain pointers and sizes, and says
  * for each pointer whether it is host or device memory.  All device work is

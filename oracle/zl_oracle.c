@@ -17,8 +17,8 @@
  * Result convention, shared by every function below so that they can be
  * compared bit for bit:
  *   wait    = min over all R^n choices of d_Z
- *   barrier = the smallest max(Z) among the minimisers ("the first minimum
- *             d_Z is selected", Fig. 3 caption; strict '<' in Algorithm 2)
+ *   barrier = the smallest max(Z) among the minimisers (of equal minima the
+ *             first one found wins: Fig. 3's caption; strict '<' in Algorithm 2)
  *   idx[p]  = the largest 0-based index i with M[p][i] <= barrier
  *             (a worker that finishes exactly at the barrier does not wait;
  *             this is the lexicographically largest minimiser with that barrier)
