@@ -68,16 +68,18 @@ zl_status zl_check_canaries(zl_handle *h, int32_t *buffers, int32_t *damaged);
  * copy, is compared with the extent of its buffer first; an index out of range is not used (the access is
  * skipped, nothing traps) and the first such event is recorded.  zl_debug_report waits for the device, copies the
  * record to h_record[0..3] (host) and clears it: [0] a code naming the access (0: no violation since the last
- * report), [1] the CTA, [2], [3] the low and high word of the offending index.  Covers the two kernels of
- * the RANGE filter route (k_range_head, k_range_filter).
+ * report), [1] the CTA, [2], [3] the low and high word of the offending index.  Covers the kernels of the
+ * RANGE filter route that every call runs (k_range_head, k_filter / k_filter_arith, k_tail) and their ring variants.
  */
 zl_status zl_debug_report(zl_handle *h, uint32_t *h_record);
 
 /*
- * With the same flag k_range_head also notes the GPU's nanosecond clock at its phase boundaries: for each of the
- * first `ctas` CTAs of the handle's last call, 16 values (0 where a boundary was not passed): [0] start, [1] columns
+ * With the same flag the kernels of the RANGE filter route also note the GPU's nanosecond clock at their phase boundaries.
+ * Records of 16 values: first k_range_head's, one per CTA, for each of the first `ctas` CTAs of the handle's last call (0 where a boundary was not passed): [0] start, [1] columns
  * done, [2] summary, [11] requests written, [12] slow rows walked, [13] partial table done, [3] before and [4] after
- * the cluster barrier, [5] merged table written.  h_stamps: host, ctas * 16 uint64.  Synchronises.
+ * the cluster barrier, [5] merged table written, [6]..[9] the last kernel's CTA of the same index (start, dependency wait over, flags read, end);
+ * behind max(max_batch, 8 x SMs) such records follow the ring variants' filter CTAs ([0] start, [1] table loaded, [2] pass done).
+ * h_stamps: host, ctas * 16 uint64.  Synchronises.
  */
 zl_status zl_debug_stamps(zl_handle *h, int32_t ctas, uint64_t *h_stamps);
 
@@ -86,7 +88,7 @@ zl_status zl_debug_stamps(zl_handle *h, int32_t ctas, uint64_t *h_stamps);
  * "segments" (time segments per instance, >= 1), "round_factor" (percent of the
  * nominal elements per round), "no_filter" (1: neither the RANGE filter route nor the bucket
  * route nor the one-launch route of small instances is used; every instance is swept by time segments), "no_small" (1: small instances do not take the one-launch route but the one larger instances of the objective would), "max_rounds" (rounds a time segment of the segment sweep may take before its instance ends with ZL_ERR_TIMEOUT; 0: the bound that follows from the input's size), "tail_cap" (a power of two, 64..2048: survivors the checked tail kernel has room for), "filter_threads" / "filter_rows" (CTA size and rows per CTA of the
- * filter pass), "cluster" (CTAs per instance of the first kernel of the RANGE filter route, a power of two up to 8), "filter_stages" (ring slots per warp, 2..7), "filter_bulk" (1: chunks of a row arrive by one bulk-copy request each, 2: in 16-byte pieces copied by every lane; default: bulk requests for whole rows, pieces for the prefixes of the early stop), "checks_off" (1: a handle created with ZL_FLAG_DEBUG_CHECKS runs the unchecked kernels but still records the clock stamps), "filter_round" (a row is requested up to its estimate rounded up to this many timestamps; power of two, 2..1024; from 128 on it is also the ring slot size of the cluster kernel), "prologue_threads" / "tail_threads" (CTA sizes of those kernels), "pdl_off" (bit k: launch the k-th kernel of the chain only after its predecessor has
+ * filter pass), "cluster" (CTAs per instance of the first kernel of the RANGE filter route, a power of two up to 8), "filter_stages" (ring slots per warp, 2..7), "filter_bulk" (the ring variants of the filter and tail kernels - 1: chunks of a row arrive by one bulk-copy request each, counted on an mbarrier; 2: in 16-byte pieces copied by every lane; 0, the default: the kernels of filter.cu, which are the faster ones on every workload measured), "checks_off" (1: a handle created with ZL_FLAG_DEBUG_CHECKS runs the unchecked kernels but still records the clock stamps), "filter_round" (a row is requested up to its estimate rounded up to this many timestamps; power of two, 2..1024; from 128 on it is also the ring slot size of the bulk-copy variant), "prologue_threads" / "tail_threads" (CTA sizes of those kernels), "pdl_off" (bit k: launch the k-th kernel of the chain only after its predecessor has
  * finished instead of scheduling it early).  0 restores the built-in choice. */
 zl_status zl_set_option(zl_handle *h, const char *key, int32_t value);
 
