@@ -232,7 +232,7 @@ zl_status zl_destroy(zl_handle *h);
 /* Queries (host side). */
 const char *zl_status_string(zl_status s);
 size_t   zl_workspace_bytes(const zl_handle *h);      /* device scratch held by the handle      */
-int32_t  zl_launches_per_call(const zl_handle *h);    /* kernels one zl_select_batched enqueues  */
+int32_t  zl_launches_per_call(const zl_handle *h);    /* kernels the next zl_select_batched enqueues */
 int32_t  zl_segments_per_instance(const zl_handle *h, int32_t B);
 int32_t  zl_route(const zl_handle *h);                /* route of the handle's calls: 0 segment sweep only, 1 RANGE filter route, 2 bucket route, 3 one launch (small instances) */
 int32_t  zl_max_workers(void);                        /* largest supported n                     */

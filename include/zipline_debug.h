@@ -87,7 +87,7 @@ zl_status zl_debug_stamps(zl_handle *h, int32_t ctas, uint64_t *h_stamps);
  * key: "threads" (128..1024, power of two), "lanes_per_row" (1..32, power of two),
  * "segments" (time segments per instance, >= 1), "round_factor" (percent of the
  * nominal elements per round), "no_filter" (1: neither the RANGE filter route nor the bucket
- * route nor the one-launch route of small instances is used; every instance is swept by time segments), "no_small" (1: small instances do not take the one-launch route but the one larger instances of the objective would), "max_rounds" (rounds a time segment of the segment sweep may take before its instance ends with ZL_ERR_TIMEOUT; 0: the bound that follows from the input's size), "tail_cap" (a power of two, 64..2048: survivors the checked tail kernel has room for), "filter_threads" / "filter_rows" (CTA size and rows per CTA of the
+ * route nor the one-launch route of small instances is used; every instance is swept by time segments), "rest_split" (RANGE filter route, what the tail kernel leaves undone: 1 a kernel per phase, 2 the single last kernel, 0 by the shape), "no_small" (1: small instances do not take the one-launch route but the one larger instances of the objective would), "max_rounds" (rounds a time segment of the segment sweep may take before its instance ends with ZL_ERR_TIMEOUT; 0: the bound that follows from the input's size), "tail_cap" (a power of two, 64..2048: survivors the checked tail kernel has room for), "filter_threads" / "filter_rows" (CTA size and rows per CTA of the
  * filter pass), "cluster" (CTAs per instance of the first kernel of the RANGE filter route, a power of two up to 8), "filter_stages" (ring slots per warp, 2..7), "filter_bulk" (the ring variants of the filter and tail kernels - 1: chunks of a row arrive by one bulk-copy request each, counted on an mbarrier; 2: in 16-byte pieces copied by every lane; 0, the default: the kernels of filter.cu, which are the faster ones on every workload measured), "checks_off" (1: a handle created with ZL_FLAG_DEBUG_CHECKS runs the unchecked kernels but still records the clock stamps), "filter_round" (a row is requested up to its estimate rounded up to this many timestamps; power of two, 2..1024; from 128 on it is also the ring slot size of the bulk-copy variant), "prologue_threads" / "tail_threads" (CTA sizes of those kernels), "pdl_off" (bit k: launch the k-th kernel of the chain only after its predecessor has
  * finished instead of scheduling it early).  0 restores the built-in choice. */
 zl_status zl_set_option(zl_handle *h, const char *key, int32_t value);

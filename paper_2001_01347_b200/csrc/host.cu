@@ -43,7 +43,7 @@ struct zl_handle {
     cudaStream_t s_stream;
     size_t staging_bytes;
     // options (0 = automatic)
-    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round, opt_cluster, opt_filter_stages, opt_checks_off, opt_filter_bulk, opt_tail_cap, opt_max_rounds, opt_no_small;
+    int opt_threads, opt_lanes, opt_segments, opt_round_factor, opt_no_filter, opt_filter_threads, opt_filter_rows, opt_pdl_off, opt_prologue_threads, opt_tail_threads, opt_filter_round, opt_cluster, opt_filter_stages, opt_checks_off, opt_filter_bulk, opt_tail_cap, opt_max_rounds, opt_no_small, opt_rest_split;
     int epoch;               // calls so far: the two sets of per-call flags alternate
     int last_cuda_error;
     int launches;
@@ -53,6 +53,9 @@ struct zl_handle {
     // ZL_FLAG_DEBUG_CHECKS: every scratch buffer ends in CANARY_BYTES bytes of a fixed pattern that no kernel may touch
     unsigned char *canary[24];
     int ncanary;
+    // RANGE filter route: one word of pinned host memory that the last kernel of a call writes (did some instance have
+    // more survivors than one CTA finishes?); the next call reads it, without waiting, to choose the form of its last stage
+    uint32_t *h_hint, *d_hint;
 };
 
 namespace {
@@ -69,7 +72,7 @@ constexpr int CANARY_BYTE = 0xC5;
 // route or plain segment sweep only).
 // RANGE filter route: from this many timestamps an instance on, what the filter and tail kernels leave undone goes
 // through kernels of its own per phase instead of the single last kernel.
-static bool range_rest_split(int n, int R) { return (long long)n * R >= (1LL << 21); }
+static bool range_rest_split(int n, int R, int forced) { return forced ? forced == 1 : (long long)n * R >= (1LL << 21); }
 
 template <class SRC>
 void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_t *ev, const SRC src) {
@@ -103,7 +106,7 @@ void enqueue(const Pipeline &q, const LaunchPlan &p, cudaStream_t st, cudaEvent_
             zl::enqueue_filter(q, fb, st, ev ? ev[2] : nullptr, src);
         }
         if (ev) cudaEventRecord(ev[3], st);
-        if (!range_rest_split(q.n, q.R)) {
+        if (!range_rest_split(q.n, q.R, q.rest_split)) {
             // everything the two kernels left undone, and the outputs, in one more launch
             zl::enqueue_range_rest(q, fb, p, st, src);
             if (ev) cudaEventRecord(ev[4], st);
@@ -271,7 +274,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
         // the fused kernel runs up to max(max_batch, 8 x SMs) CTAs, each with a record of partial results and a partial table
         const size_t ctas = std::max<size_t>(mb, (size_t)h->num_sms * 8);
         const size_t sizes[12] = {mb * f.cells * 4, mb * cfg->n_workers * 4, mb * f.fcells * 4, std::max<size_t>(mb * cfg->n_workers, ctas) * 4,
-                                  mb * (size_t)f.list1cap * 8, mb * f.nbk * 4, mb * f.nbk * f.capb * 8, mb * tiles * 4, 64,
+                                  mb * (size_t)f.list1cap * 8, mb * f.nbk * 4, mb * f.nbk * f.capb * 8, mb * tiles * 4, 128,
                                   ctas * 4 * 8, ctas * f.cells * 4, mb * 4};
         void **ptrs[12] = {(void **)&f.table, (void **)&f.rowhint, (void **)&f.cellmax, (void **)&f.rcnt,
                            (void **)&f.list1, (void **)&f.bcnt, (void **)&f.list2, (void **)&f.tilemax, (void **)&f.flags,
@@ -281,7 +284,11 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
             if (e == cudaSuccess) e = alloc(ptrs[i], sizes[i]);
             filter_b += sizes[i];
         }
-        if (e == cudaSuccess) e = cudaMemset(f.flags, 0, 64);
+        if (e == cudaSuccess) e = cudaMemset(f.flags, 0, 128);      // two sets of eight per-call words, then words that outlive a call
+        if (e == cudaSuccess) e = cudaHostAlloc((void **)&h->h_hint, 64, cudaHostAllocMapped);
+        if (e == cudaSuccess) { memset(h->h_hint, 0, 64); e = cudaHostGetDevicePointer((void **)&h->d_hint, h->h_hint, 0); }
+        f.hint = h->d_hint;
+        f.hint_last = e == cudaSuccess ? f.flags + 16 : nullptr;
         if (cfg->flags & ZL_FLAG_DEBUG_CHECKS) {
             // the violation record, then 16 clock stamps per CTA of the head kernel and of the filter kernel
             const size_t dbg_b = 64 + (ctas + mb * ((size_t)cfg->n_workers + 1) / 2 + 1) * 16 * 8;
@@ -328,6 +335,7 @@ zl_status zl_create(const zl_config *cfg, zl_handle **out) {
     if (e != cudaSuccess) {
         zl_status st = cuda_fail(nullptr, e);
         cudaFree(h->d_meta); cudaFree(h->d_seg); cudaFree(h->d_pred);
+        if (h->h_hint) cudaFreeHost(h->h_hint);
         cudaFree(h->fb.table); cudaFree(h->fb.rowhint); cudaFree(h->fb.cellmax); cudaFree(h->fb.rcnt);
         cudaFree(h->fb.list1); cudaFree(h->fb.bcnt); cudaFree(h->fb.list2); cudaFree(h->fb.tilemax); cudaFree(h->fb.flags);
         cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab); cudaFree(h->fb.part); cudaFree(h->fb.ptab); cudaFree(h->fb.dbg); cudaFree(h->fb.done);
@@ -399,6 +407,7 @@ zl_status zl_destroy(zl_handle *h) {
     cudaFree(h->fb.bnd); cudaFree(h->fb.cellacc); cudaFree(h->fb.itab); cudaFree(h->fb.part); cudaFree(h->fb.ptab); cudaFree(h->fb.dbg); cudaFree(h->fb.done);
     cudaFree(h->s_ts); cudaFree(h->s_idx); cudaFree(h->s_barrier); cudaFree(h->s_wait); cudaFree(h->s_status);
     if (h->s_stream) cudaStreamDestroy(h->s_stream);
+    if (h->h_hint) cudaFreeHost(h->h_hint);
     zl_profile_end(h);
     delete h;
     return ZL_OK;
@@ -427,6 +436,9 @@ zl_status zl_set_option(zl_handle *h, const char *key, int32_t value) {
     } else if (!strcmp(key, "filter_bulk")) {
         if (value > 2) return ZL_ERR_INVALID_ARG;
         h->opt_filter_bulk = value;
+    } else if (!strcmp(key, "rest_split")) {
+        if (value > 2) return ZL_ERR_INVALID_ARG;
+        h->opt_rest_split = value;                  // RANGE filter route, what the tail kernel leaves: 1 a kernel per phase, 2 the single last kernel
     } else if (!strcmp(key, "no_small")) {
         h->opt_no_small = value != 0;               // small instances take the route larger ones would (bucket route)
     } else if (!strcmp(key, "max_rounds")) {
@@ -468,12 +480,20 @@ static bool small_route(const zl_handle *h) {
            !h->opt_no_filter && !h->opt_no_small && !(h->cfg.flags & ZL_FLAG_FORCE_FILTER);
 }
 
+// The form of the RANGE filter route's last stage for the handle's next call: a kernel per phase when the shape is large,
+// or when the previous call (as far as its word has arrived: the read does not wait) had instances with many survivors.
+static int rest_split_now(const zl_handle *h) {
+    if (h->opt_rest_split) return h->opt_rest_split == 1;
+    if (range_rest_split(h->cfg.n_workers, h->cfg.lookahead_R, 0)) return 1;
+    return h->h_hint && *(volatile const uint32_t *)h->h_hint != 0;
+}
+
 int32_t zl_launches_per_call(const zl_handle *h) {
     if (!h) return 0;
     if (small_route(h)) return 1;
     const bool filter = h->cfg.objective == ZL_OBJ_RANGE && !h->opt_no_filter && h->fb.table != nullptr;
     const bool sumfast = !filter && !h->opt_no_filter && h->fb.scap != 0;
-    return (filter ? (range_rest_split(h->cfg.n_workers, h->cfg.lookahead_R) ? 9 : 4) : 3) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
+    return (filter ? (rest_split_now(h) ? 9 : 4) : 3) + (sumfast ? (h->fb.scells ? 3 : 2) : 0) + ((h->cfg.flags & ZL_FLAG_CHECK_SORTED) ? 1 : 0);
 }
 int32_t zl_route(const zl_handle *h) {
     if (!h || h->opt_no_filter) return 0;
@@ -506,7 +526,7 @@ zl_status zl_select_batched(zl_handle *h, const int64_t *d_ts, int32_t B, int32_
     q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
     if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
     q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
-    q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds; q.small = small_route(h) ? 1 : 0;
+    q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds; q.small = small_route(h) ? 1 : 0; q.rest_split = rest_split_now(h) ? 1 : 2;
     if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
         uint32_t *base = h->fb.flags;
         q.fb.flags = base + 8 * (h->epoch & 1);
@@ -599,7 +619,7 @@ zl_status zl_predict_select_batched(zl_handle *h, const int64_t *d_last, const i
         q.prologue_threads = h->opt_prologue_threads; q.tail_threads = h->opt_tail_threads;
         if (h->opt_no_filter) { q.fb.table = nullptr; q.fb.scap = 0; }
         q.cluster = h->opt_cluster; q.filter_stages = h->opt_filter_stages;
-        q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds; q.small = small_route(h) ? 1 : 0;
+        q.checks_off = h->opt_checks_off; q.filter_bulk = h->opt_filter_bulk; q.tail_cap = h->opt_tail_cap; q.rest_per_sm = 0; q.max_rounds = h->opt_max_rounds; q.small = small_route(h) ? 1 : 0; q.rest_split = rest_split_now(h) ? 1 : 2;
         if (q.fb.flags) {                           // the two sets of per-call flags alternate; a call zeroes the next call's set
             uint32_t *base = h->fb.flags;
             q.fb.flags = base + 8 * (h->epoch & 1);
@@ -725,7 +745,7 @@ zl_status zl_select_batched_noalloc(int32_t n_workers, int32_t lookahead_R, int3
     q.ts = d_ts; q.B = B; q.n = n_workers; q.R = lookahead_R; q.objective = objective; q.flags = flags; q.num_sms = tmp.num_sms;
     q.meta = meta; q.seg = seg; q.nres = p.nseg;
     memset(&q.fb, 0, sizeof(q.fb));
-    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0; q.cluster = q.filter_stages = 0; q.checks_off = 0; q.filter_bulk = 0; q.tail_cap = 0; q.rest_per_sm = 0; q.max_rounds = 0; q.small = (long long)n_workers * lookahead_R <= zl::SMALL_MAX && B <= 4 * std::max(1, tmp.num_sms) ? 1 : 0;
+    q.filter_threads = q.filter_rows = q.filter_round = 0; q.pdl_off = 0; q.prologue_threads = q.tail_threads = 0; q.cluster = q.filter_stages = 0; q.checks_off = 0; q.filter_bulk = 0; q.tail_cap = 0; q.rest_per_sm = 0; q.max_rounds = 0; q.rest_split = 0; q.small = (long long)n_workers * lookahead_R <= zl::SMALL_MAX && B <= 4 * std::max(1, tmp.num_sms) ? 1 : 0;
     q.idx = d_idx; q.barrier = d_barrier; q.wait = d_wait; q.status = d_status;
     enqueue(q, p, (cudaStream_t)cuda_stream, nullptr, zl::MatBatch{d_ts});
     return cudaGetLastError() == cudaSuccess ? ZL_OK : ZL_ERR_CUDA;

@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(REST_THREADS) k_range_rest(const SRC src, cons
     unsigned int k = 0;
     bool ok = true;
     const uint4 fl4 = __ldcg(reinterpret_cast<const uint4 *>(F.flags));        // [0] .. [3] together
+    if (F.hint && blockIdx.x == 0 && threadIdx.x == 0) note_hint(F, fl4.x != 0u);   // for the host's next call
     if ((fl4.x | fl4.y | fl4.z) == 0) return;                     // the tail kernel finished every instance of the call
     const uint64_t fl = ((uint64_t)fl4.y << 32) | fl4.x;
     // in the same round of loads: what the outputs of the warp's first rows need (read again below if a phase ran)

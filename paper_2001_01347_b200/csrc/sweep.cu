@@ -24,6 +24,7 @@ __global__ void __launch_bounds__(256) k_finalize(const SRC src, int B, int n, i
     // (Input, read before the wait: this is not the call's first kernel, and it starts only when every CTA of its predecessor
     // has exited, i.e. has passed its own wait, so whatever produced the input before the call had completed by then.)
     grid_dep_wait();
+    if (filter == 1 && F.hint && blockIdx.x == 0 && threadIdx.x == 0) note_hint(F, F.flags[0] != 0u);   // for the host's next call
     if (filter == 1 && F.flags[2] == 0) return;                   // the tail kernel finished every instance of the call
     finalize_all(src, B, n, R, nseg, F, nres, objective, filter, meta, seg, idx, barrier, wait, status, 0u, &first);
 }

@@ -31,6 +31,7 @@ struct Pipeline {
     int prologue_threads, tail_threads;                           // 0: automatic
     int cluster, filter_stages, filter_bulk;                      // 0: automatic (cluster: CTAs per instance of k_range_head; filter_bulk: 1 copy engine, 2 per-lane copies)
     int tail_cap;                                                 // 0: default; else survivors the finishing CTA of the filter kernel has room for
+    int rest_split;                                               // RANGE filter route's last stage: 0 by shape, 1 a kernel per phase, 2 the single kernel
     int small;                                                    // 1: the one-launch route (instances of a few thousand timestamps)
     int max_rounds;                                               // 0: automatic; else the segment sweep's round limit
     int rest_per_sm;                                              // CTAs of k_range_rest resident per SM (0: ask the runtime)

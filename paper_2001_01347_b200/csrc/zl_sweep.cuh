@@ -248,6 +248,12 @@ __device__ void sweep_items(const SweepParams &P, const SRC &src, SweepShared &s
     }
 }
 
+// The word the host reads before its next call (pinned host memory): written across the bus only when it changes.
+__device__ __forceinline__ void note_hint(const FilterBufs &F, bool many) {
+    const uint32_t v = many ? 1u : 0u;
+    if (*F.hint_last != v) { *F.hint_last = v; *F.hint = v; }
+}
+
 // ------------------------------------------------------------------------------ finalize
 // The final step for 32 consecutive rows of an instance, by one warp: the minimum over the instance's partial results
 // (every warp of the instance takes it for itself: there are few of them), then the indices of the warp's rows, a row

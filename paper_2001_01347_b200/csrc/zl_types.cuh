@@ -101,6 +101,9 @@ struct FilterBufs {
                          //                   grid-wide barriers of the route's last kernel, [5] one of its barriers gave up
     uint32_t *flags_next; // [8]              the flags of the handle's next call (the two sets alternate); zeroed by this call
     uint64_t *part;      // [ctas][4]         k_range_head: per-CTA minima / maxima of the first and last column
+    uint32_t *hint;      // [1]               pinned host memory (device address), or nullptr: the call's last kernel notes here whether some
+                         //                   instance had more survivors than one CTA finishes
+    uint32_t *hint_last; // [1]               device: what was last written to `hint` (the word is written only when it changes)
     uint32_t *done;      // [B]               blocks of the filter pass that have finished, per instance (in the end: how many it had)
     uint32_t *ptab;      // [ctas][cells]     k_range_head: per-CTA partial filter tables
     int32_t maxctas;     //                   CTAs k_range_head's per-CTA records have room for

@@ -144,6 +144,36 @@ def test_filter_route_rows_far_from_arithmetic(variant):
             h.destroy()
 
 
+def test_many_survivor_phases_in_one_kernel_and_in_kernels_of_their_own():
+    # instances with more survivors than one CTA finishes: the phases behind the tail kernel run inside the route's single
+    # last kernel (grid-wide barriers between them) or as a kernel each; both must give the oracle's result
+    rng = np.random.default_rng(303)
+    shapes = [(100, 150, 40, 0), (128, 256, 64, 1), (257, 65, 9, 2)]
+    for n, R, B, kind in shapes:
+        if kind == 0:
+            ts = zi.generate(zi.CONFIGS["c2"].with_(B=B, n=n, R=R))
+        elif kind == 1:      # a homogeneous cluster: every row is slow, most elements raise the running maximum
+            v = rng.integers(99_000, 101_000, size=(B, n, 1))
+            ts = (rng.integers(0, 100_000, size=(B, n, 1)) + np.cumsum(v + rng.integers(0, 50, size=(B, n, R)), axis=2)).astype(np.int64)
+        else:
+            ts = (rng.integers(0, 5, size=(B, n, 1)) + np.cumsum(rng.integers(0, 3, size=(B, n, R)), axis=2)).astype(np.int64)
+        for mode in (1, 2):
+            got = gpu_select(ts, 0, options={"rest_split": mode})
+            assert_same(ts, 0, got)
+    # left to itself a handle takes the form from what its previous call met: a kernel per phase after a call with such
+    # instances, the single kernel again after a call without
+    heavy = ts_heavy = (rng.integers(0, 100_000, size=(8, 128, 1)) + np.cumsum(100_000 + rng.integers(0, 50, size=(8, 128, 256)), axis=2)).astype(np.int64)
+    light = zi.generate(zi.CONFIGS["c3"].with_(B=8))
+    h = zl.ZipLine(128, 256, 8, 0)
+    assert h.launches_per_call == 4
+    for ts, after in ((heavy, 9), (heavy, 9), (light, 4), (light, 4), (heavy, 9)):
+        sel = h.select_batched(torch.from_numpy(ts).cuda())
+        torch.cuda.synchronize()
+        assert_same(ts, 0, (sel.idx.cpu().numpy(), sel.barrier.cpu().numpy(), sel.wait.cpu().numpy(), sel.status.cpu().numpy()))
+        assert h.launches_per_call == after
+    h.destroy()
+
+
 def test_filter_route_dense_ties_just_above_the_single_batch_size():
     # 256 instances of slightly more than 4096 timestamps with many equal values: the filter route's natural smallest shapes
     rng = np.random.default_rng(301)
