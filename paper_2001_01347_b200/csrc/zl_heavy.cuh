@@ -6,6 +6,8 @@
 
 namespace zl {
 
+constexpr int REFINE_ILP = 8;           // survivors a thread of the refinement has in flight
+
 // ------------------------------------------------------------------------------ refinement (RANGE)
 // The per-cell maxima of the filter pass give G exactly at every fine cell start (the survivors contain
 // every element that ever raises the running maximum): heavy_cellscan turns cellmax, in place, into its
@@ -77,19 +79,19 @@ static __device__ void heavy_refine(InstMeta *meta, const FilterBufs &F, int B) 
         uint64_t *dst = F.list2 + (size_t)b * F.nbk * F.capb;
         unsigned kept = 0;
         bool over = false;
-        // four elements a step, so that four list loads and then four table look-ups are in flight together
-        for (uint32_t i0 = tid; i0 < m; i0 += 4 * nt) {
-            uint64_t w[4];
-            uint32_t c[4], gv[4];
+        // REFINE_ILP elements a step, so that as many list loads and then as many table look-ups are in flight together
+        for (uint32_t i0 = tid; i0 < m; i0 += REFINE_ILP * nt) {
+            uint64_t w[REFINE_ILP];
+            uint32_t c[REFINE_ILP], gv[REFINE_ILP];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) { const uint32_t i = i0 + k * nt; w[k] = i < m ? src[i] : 0ull; }
+            for (int k = 0; k < REFINE_ILP; ++k) { const uint32_t i = i0 + k * nt; w[k] = i < m ? src[i] : 0ull; }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < REFINE_ILP; ++k) {
                 c[k] = w[k] ? cell_of((uint32_t)(w[k] >> 32), M.fscale) : 0u;
                 gv[k] = __ldcg(g + c[k]);
             }
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
+            for (int k = 0; k < REFINE_ILP; ++k) {
                 const uint32_t T = (uint32_t)(w[k] >> 32), nx = (uint32_t)w[k];
                 if (w[k] && nx > max(T, gv[k])) {
                     const uint32_t bk = c[k] >> cpb_shift;
