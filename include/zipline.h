@@ -197,18 +197,21 @@ zl_status zl_trace_batched(const int64_t *d_ts, int32_t B, int32_t n, int32_t R,
  * point keeps the scratch it needs (per-instance summaries and per-segment partial
  * results) in a fixed array compiled into the library instead, zl_noalloc_scratch_bytes()
  * bytes (about 400 KB) that every GPU using the library holds until the process exits.
- * It calls no cudaMalloc, cudaFree or other allocating routine.  It always runs the
- * segment sweep; the faster filter route of the RANGE objective needs buffers of about
- * the size of the input and is only available through a handle.
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  Instances of at most
+ * 4096 timestamps in batches of up to four per SM run the one-launch kernel, which needs
+ * no scratch at all; everything else runs the segment sweep.  The faster filter route of
+ * the RANGE objective needs buffers of about the size of the input and is only available
+ * through a handle.
  *
  * Arguments are those of zl_create's configuration (n_workers, lookahead_R, objective,
  * flags) followed by those of zl_select_batched, with the same meaning, layout and
  * ownership; the device is the calling thread's current CUDA device, which must own
  * every buffer.  Asynchronous on cuda_stream.
  *
- * Limits: B <= zl_noalloc_max_batch() (256), and B times the number of time segments
- * the launch planner picks must fit the array; larger requests return
- * ZL_ERR_UNSUPPORTED with a message on stderr and launch nothing.
+ * Limits: B <= zl_noalloc_max_batch() (256); a larger batch returns ZL_ERR_UNSUPPORTED
+ * with a message on stderr and launches nothing.  (B times the number of time segments
+ * must also fit the array; the built-in launch planner never picks that many, the test
+ * is a guard.)
  *
  * First call on a device: looks up the array's device address and raises the sweep
  * kernel's shared-memory limit.  Make that first call outside any stream capture.
